@@ -1,0 +1,183 @@
+/*
+ * sdfp.h — C ABI of the SDFP speculative-decode library for NVIDIA B200 (sm_100a).
+ *
+ * The library runs the online stage of SDFP (Algorithm 1, Stage B, "Speculative
+ * Decoding with Pruned Draft Model"; Section II-A for the accept/reject rule):
+ * a Llama-style decoder drafts k tokens with a subset of its own layers, the
+ * full stack verifies k+1 positions in one pass, the longest accepted prefix
+ * plus one corrected/bonus token is committed, and both KV caches roll back.
+ *
+ * Conventions
+ *   - Every function returns 0 on success or a negative sdfp_status; nothing is
+ *     thrown, nothing aborts.  sdfp_last_error() gives the text of the last
+ *     failure on that context (or of the last failed sdfp_create when ctx is NULL).
+ *   - "device" pointers are CUDA global-memory addresses valid on the device
+ *     that is current when sdfp_create is called; "host" pointers are ordinary
+ *     host memory.  The library never frees or writes caller-owned memory
+ *     except the documented outputs.
+ *   - All work is issued on the CUDA stream given to sdfp_create (borrowed, the
+ *     caller keeps ownership; NULL = the legacy default stream).
+ *   - Deterministic: same config, weights, mask, prompts, k, temperature and
+ *     seed give bit-identical outputs, and a sequence's tokens do not depend on
+ *     what else is in the batch nor on how many rows a pass carries.
+ *   - There is no CPU fallback: without a usable CUDA device every entry point
+ *     that computes fails with SDFP_ECUDA.
+ */
+#ifndef SDFP_H_
+#define SDFP_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct sdfp_ctx sdfp_ctx; /* opaque, library-owned */
+
+typedef enum {
+  SDFP_OK = 0,
+  SDFP_EINVAL = -1, /* bad argument or unsupported shape            */
+  SDFP_ENOMEM = -2, /* device or host allocation failed             */
+  SDFP_ECUDA = -3,  /* a CUDA call failed (text in sdfp_last_error) */
+  SDFP_ESTATE = -4  /* call not valid in the context's state        */
+} sdfp_status;
+
+typedef enum { SDFP_F32 = 0, SDFP_BF16 = 1 } sdfp_dtype;
+
+/* sdfp_config.flags */
+#define SDFP_FLAG_NO_GRAPH 1u /* launch kernels directly instead of replaying CUDA graphs    */
+#define SDFP_FLAG_NO_PDL 2u   /* no programmatic dependent launch between consecutive kernels */
+#define SDFP_FLAG_FMA_GEMM 4u /* bf16 models: CUDA-core FMA GEMM instead of the tensor path  */
+
+/*
+ * Model and capacity description.  The decoder is the LLaMA-2 architecture the
+ * paper evaluates (Section IV-A): RMSNorm(eps inside the root), rotary
+ * embeddings on pairs (i, i + head_dim/2) with base rope_theta, multi-head
+ * causal attention (n_kv_heads == n_heads), SwiGLU FFN, untied lm-head, no bias.
+ * Requirements: d_model == n_heads*head_dim; head_dim in {64, 128}; d_model,
+ * d_ffn and vocab multiples of 16; max_batch*(k_max+1) <= 64.
+ */
+typedef struct {
+  int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
+  float rms_eps, rope_theta;
+  int32_t max_seq;   /* KV-cache capacity per sequence, tokens              */
+  int32_t max_batch; /* sequences per sdfp_generate call                    */
+  int32_t k_max;     /* largest draft length k that will be requested       */
+  int32_t dtype;     /* sdfp_dtype: storage type of weights and of the KV cache */
+  int32_t eos_id;    /* < 0: never stop on a token                          */
+  uint32_t flags;
+} sdfp_config;
+
+/*
+ * Weights: DEVICE pointers, every matrix row-major [out_features, in_features]
+ * in the storage type of the config.  The per-layer members point to HOST
+ * arrays of n_layers device pointers.  sdfp_create re-packs everything into
+ * library-owned buffers (fused QKV, interleaved gate/up, tensor-core fragment
+ * order) and does not keep the caller's pointers: the caller may free its
+ * tensors after sdfp_create returns.
+ */
+typedef struct {
+  const void *tok_embed;  /* [vocab, d_model] */
+  const void *final_norm; /* [d_model]        */
+  const void *lm_head;    /* [vocab, d_model] */
+  const void *const *wq, *const *wk, *const *wv, *const *wo; /* [d_model, d_model] each */
+  const void *const *w_gate, *const *w_up;                   /* [d_ffn, d_model]        */
+  const void *const *w_down;                                 /* [d_model, d_ffn]        */
+  const void *const *attn_norm, *const *ffn_norm;            /* [d_model]               */
+} sdfp_weights;
+
+/* One speculative round of one sequence (Algorithm 1, loop body). */
+typedef struct {
+  int32_t drafted;   /* k                                                    */
+  int32_t accepted;  /* j = length of the accepted prefix (Eq. 2), 0..k      */
+  int32_t committed; /* tokens appended this round after truncation, <= j+1  */
+} sdfp_round_stat;
+
+/* Timing and traffic of the last sdfp_generate call (CUDA events on the stream). */
+typedef struct {
+  float prefill_ms;         /* prompt pass(es) of target and draft                     */
+  float decode_ms;          /* first round's first kernel .. last round's last kernel  */
+  int32_t n_rounds;         /* rounds (speculative) or steps (k = 0)                   */
+  int32_t n_draft_passes;   /* draft forward passes in the decode phase                */
+  int32_t n_target_passes;  /* verify (or autoregressive) passes in the decode phase   */
+  int64_t kernel_launches;  /* kernels of this library launched in the decode phase    */
+  int64_t weight_bytes;     /* weight bytes the decode-phase passes had to read        */
+  int64_t kv_bytes;         /* KV-cache bytes read + written in the decode phase       */
+  int64_t tokens_committed; /* over all sequences                                      */
+} sdfp_timing;
+
+/*
+ * Create a context: validates the config, packs the weights, allocates both KV
+ * caches (target: all layers; draft: its own cache for the kept layers, Section
+ * III-C "architecture-compatible") and all scratch.  `cuda_stream` is a
+ * cudaStream_t.  The draft initially keeps every layer.
+ */
+int sdfp_create(const sdfp_config *cfg, const sdfp_weights *w, void *cuda_stream, sdfp_ctx **out);
+
+/*
+ * Select the draft model (Algorithm 1: "construct draft model by removing
+ * layers in P"): keep_mask is a HOST array of n_layers bytes, 1 = the draft runs
+ * the layer, 0 = the layer is the identity for the draft.  At least one layer
+ * must be kept.  Takes effect at the next sdfp_generate.
+ */
+int sdfp_set_draft_layers(sdfp_ctx *ctx, const uint8_t *keep_mask);
+
+/*
+ * Generate (Algorithm 1, Stage B).  Synchronous: returns when the outputs are
+ * in host memory.
+ *   prompts     host int32 [batch, prompt_len], ids in [0, vocab); prompt_len >= 1
+ *   k           draft length per round, 1..k_max; 0 = plain autoregressive decoding
+ *               with the full model (the "vanilla" baseline of Table I)
+ *   max_new     tokens to produce per sequence (fewer if eos_id is produced)
+ *   temperature 0 = greedy (accept iff the draft token is the target's argmax, ties
+ *               to the lowest id); > 0 = sampling from softmax(logits/temperature)
+ *               with the accept rule of Eq. 2 and residual resampling (Eq. 3 read as
+ *               normalised max(0, p − q))
+ *   seed        key of the Philox4x32-10 streams (sampling only)
+ *   out_tokens  host int32 [batch, max_new]; entries beyond out_len[b] are −1
+ *   out_len     host int32 [batch]
+ *   stats       host [max_rounds, batch] or NULL; round r of sequence b at
+ *               stats[r*batch + b]; sequences that were already finished in a
+ *               round report {0,0,0}
+ *   n_rounds    host int32, rounds executed (may be NULL)
+ * Fails with SDFP_EINVAL when prompt_len + max_new + k + 1 > max_seq,
+ * batch > max_batch, k > k_max, temperature < 0 or a pointer is NULL.
+ */
+int sdfp_generate(sdfp_ctx *ctx, const int32_t *prompts, int32_t batch, int32_t prompt_len,
+                  int32_t k, int32_t max_new, float temperature, uint64_t seed,
+                  int32_t *out_tokens, int32_t *out_len, sdfp_round_stat *stats,
+                  int32_t max_rounds, int32_t *n_rounds);
+
+/*
+ * Test hook: run `rows` tokens of ONE sequence at positions start.. through the
+ * target (draft == 0) or the draft (draft != 0) model on sequence slot 0,
+ * writing K/V into that model's cache from `start` on, and copy the logits
+ * [rows, vocab] (fp32) to host.  rows <= 64.  Lets a test compare logits with
+ * the oracle position by position, in chunks of any size.
+ */
+int sdfp_forward_logits(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int32_t rows,
+                        int32_t start, float *host_logits);
+
+/* Timing of the last successful sdfp_generate. */
+int sdfp_get_timing(const sdfp_ctx *ctx, sdfp_timing *out);
+
+/*
+ * Micro-benchmark hook for the roofline report: launches the library's
+ * weight-streaming linear kernel of layer `layer` (which: 0 = QKV, 1 = O,
+ * 2 = gate/up, 3 = down, 4 = lm-head) with `rows` activation rows `iters`
+ * times back to back on the context's stream, layer advancing cyclically so
+ * that consecutive launches read different weights, and returns the average
+ * duration of one launch in milliseconds (CUDA events) and the weight bytes one
+ * launch reads.  Scratch activations are used; caches are not touched.
+ */
+int sdfp_time_linear(sdfp_ctx *ctx, int32_t which, int32_t rows, int32_t iters,
+                     float *ms_per_launch, int64_t *weight_bytes_per_launch);
+
+const char *sdfp_last_error(const sdfp_ctx *ctx);
+void sdfp_destroy(sdfp_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SDFP_H_ */

@@ -1,0 +1,782 @@
+// Host engine and C ABI of the SDFP speculative-decode library (see include/sdfp.h).
+//
+// One forward pass = plan+embed, then per running layer
+//   [RMSNorm + QKV + RoPE + KV append] -> [split-KV attention] -> [O-proj + residual]
+//   -> [RMSNorm + gate/up + SwiGLU] -> [down-proj + residual],
+// then [final RMSNorm + lm-head] and a token decision.  A speculative round is
+// k draft passes (kept layers, own KV cache), one verify pass over k+1 rows (all
+// layers) and one accept/commit kernel; all lengths live on the device, so a round
+// is a fixed kernel sequence that is captured once as a CUDA graph and replayed.
+#include <cuda_runtime.h>
+
+#include <algorithm>
+#include <cmath>
+#include <cstdarg>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <new>
+#include <string>
+#include <tuple>
+#include <vector>
+
+#include "../../include/sdfp.h"
+#include "attention.cuh"
+#include "common.cuh"
+#include "linear_fma.cuh"
+#include "linear_mma.cuh"
+#include "misc_kernels.cuh"
+#include "sampling.cuh"
+
+using namespace sdfp;
+
+namespace {
+
+thread_local std::string g_create_error;
+
+struct LayerWeights {
+  void* qkv = nullptr;   // packed [3d, d]
+  void* wo = nullptr;    // packed [d, d]
+  void* gu = nullptr;    // packed [2f, d]
+  void* down = nullptr;  // packed [d, f]
+  float* attn_gain = nullptr;
+  float* ffn_gain = nullptr;
+};
+
+struct KvCache {
+  std::vector<void*> k, v;  // per layer: [max_batch][heads][max_seq][head_dim]
+};
+
+}  // namespace
+
+struct sdfp_ctx {
+  sdfp_config cfg{};
+  cudaStream_t stream = nullptr;
+  std::string err;
+  bool bf16 = false, use_mma = false, use_pdl = true, use_graph = true;
+  size_t esz = 4;  // bytes per stored element
+  int num_sms = 148;
+
+  std::vector<LayerWeights> layers;
+  void* embed = nullptr;
+  void* lm_head = nullptr;
+  float* final_gain = nullptr;
+  float *rope_cos = nullptr, *rope_sin = nullptr;
+  KvCache cache_t, cache_d;
+  std::vector<uint8_t> keep;
+
+  // activations / scratch
+  float *h = nullptr, *q = nullptr, *att = nullptr, *u = nullptr, *logits = nullptr;
+  float *part_o = nullptr, *part_ml = nullptr;
+  int* attn_counters = nullptr;
+  int n_chunks_cap = 0;
+  RowPlan plan{};
+  int *seq_tok = nullptr, *draft_tok = nullptr, *tgt_tok = nullptr, *row_argmax = nullptr, *out_tok = nullptr;
+  int* fwd_tok = nullptr;
+  float* qprob = nullptr;  // sampling: unnormalised draft probabilities [max_batch][kMaxK][vocab]
+  double* qsum = nullptr;  // [max_batch][kMaxK]
+  GenState* gs = nullptr;
+  RoundStat* stats = nullptr;
+  int stats_cap = 0;
+  int* pinned_flag = nullptr;  // host pinned: [all_done, round]
+
+  std::vector<void*> allocs;
+  struct RoundGraph {
+    cudaGraphExec_t exec;
+    long long launches;
+  };
+  std::map<std::tuple<int, int, int, int>, RoundGraph> graphs;  // (k, batch, sampled, n_chunks)
+  long long launches = 0;
+  Launcher L{};
+  bool own_stream = false;
+  sdfp_timing timing{};
+  cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
+};
+
+namespace {
+
+int fail(sdfp_ctx* c, int code, const char* fmt, ...) {
+  char buf[512];
+  va_list ap;
+  va_start(ap, fmt);
+  vsnprintf(buf, sizeof buf, fmt, ap);
+  va_end(ap);
+  if (c)
+    c->err = buf;
+  else
+    g_create_error = buf;
+  return code;
+}
+
+#define CU_OK(c, call)                                                                          \
+  do {                                                                                          \
+    cudaError_t e_ = (call);                                                                    \
+    if (e_ != cudaSuccess)                                                                      \
+      return fail((c), e_ == cudaErrorMemoryAllocation ? SDFP_ENOMEM : SDFP_ECUDA, "%s: %s", #call, \
+                  cudaGetErrorString(e_));                                                      \
+  } while (0)
+
+template <typename T>
+int dev_alloc(sdfp_ctx* c, T** p, size_t n, bool zero = false) {
+  void* q = nullptr;
+  CU_OK(c, cudaMalloc(&q, std::max<size_t>(n * sizeof(T), 16)));
+  c->allocs.push_back(q);
+  if (zero) CU_OK(c, cudaMemsetAsync(q, 0, std::max<size_t>(n * sizeof(T), 16), c->stream));
+  *p = reinterpret_cast<T*>(q);
+  return 0;
+}
+
+template <typename... KArgs, typename... Args>
+cudaError_t launch(sdfp_ctx* c, void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, Args&&... args) {
+  return launch_kernel(c->L, kernel, grid, block, smem, std::forward<Args>(args)...);
+}
+
+// ---- linear layer dispatch ---------------------------------------------------------
+
+struct LinearCall {
+  const void* w;
+  const float* x;
+  int ldx, rows, K, n_pairs;
+  const float* gain;  // non-null: RMSNorm of x with this gain first
+  EpiParams ep;
+};
+
+int linear_grid_fma(const sdfp_ctx* c, int n_pairs) {
+  const int want = (n_pairs + 7) / 8;
+  return std::max(1, std::min(want, c->num_sms * 8));
+}
+
+cudaError_t run_linear(sdfp_ctx* c, const LinearCall& lc) {
+  if (c->use_mma)
+    return launch_linear_mma(c->L, c->num_sms, lc.w, lc.x, lc.ldx, lc.rows, lc.K, lc.n_pairs, lc.gain, c->cfg.rms_eps, lc.ep);
+  const dim3 grid(linear_grid_fma(c, lc.n_pairs)), block(kFmaThreads);
+  if (c->bf16)
+    return launch(c, linear_fma_kernel<__nv_bfloat16, __nv_bfloat16>, grid, block, 0,
+                  reinterpret_cast<const __nv_bfloat16*>(lc.w), lc.x, lc.ldx, lc.rows, lc.K, lc.n_pairs, lc.gain,
+                  c->cfg.rms_eps, lc.ep);
+  return launch(c, linear_fma_kernel<float, float>, grid, block, 0, reinterpret_cast<const float*>(lc.w), lc.x,
+                lc.ldx, lc.rows, lc.K, lc.n_pairs, lc.gain, c->cfg.rms_eps, lc.ep);
+}
+
+EpiParams base_epi(const sdfp_ctx* c, int mode, float* out, int ld) {
+  EpiParams ep{};
+  ep.mode = mode;
+  ep.out = out;
+  ep.out_ld = ld;
+  ep.rope_cos = c->rope_cos;
+  ep.rope_sin = c->rope_sin;
+  ep.row_pos = c->plan.row_pos;
+  ep.row_seq = c->plan.row_seq;
+  ep.n_heads = c->cfg.n_heads;
+  ep.head_dim = c->cfg.head_dim;
+  ep.max_seq = c->cfg.max_seq;
+  return ep;
+}
+
+template <typename KT, int HD>
+cudaError_t launch_attention_t(sdfp_ctx* c, const AttnParams& ap, int n_groups) {
+  const size_t smem = attention_smem_bytes<KT, HD>();
+  return launch(c, attention_kernel<KT, HD>, dim3(ap.n_chunks, ap.n_heads, n_groups), dim3(kAttnThreads), smem, ap);
+}
+
+cudaError_t run_attention(sdfp_ctx* c, const KvCache& kv, int layer, int rows, int rows_per_seq, int n_chunks) {
+  AttnParams ap{};
+  ap.q = c->q;
+  ap.kcache = kv.k[layer];
+  ap.vcache = kv.v[layer];
+  ap.out = c->att;
+  ap.part_o = c->part_o;
+  ap.part_ml = c->part_ml;
+  ap.counters = c->attn_counters;
+  ap.row_pos = c->plan.row_pos;
+  ap.row_seq = c->plan.row_seq;
+  ap.rows_per_seq = rows_per_seq;
+  ap.n_heads = c->cfg.n_heads;
+  ap.max_seq = c->cfg.max_seq;
+  ap.n_chunks = n_chunks;
+  ap.scale = 1.0f / std::sqrt((float)c->cfg.head_dim);
+  const int n_groups = rows / rows_per_seq;
+  const bool hd128 = c->cfg.head_dim == 128;
+  if (c->bf16)
+    return hd128 ? launch_attention_t<__nv_bfloat16, 128>(c, ap, n_groups)
+                 : launch_attention_t<__nv_bfloat16, 64>(c, ap, n_groups);
+  return hd128 ? launch_attention_t<float, 128>(c, ap, n_groups) : launch_attention_t<float, 64>(c, ap, n_groups);
+}
+
+template <typename KT, int HD>
+cudaError_t configure_attention_t() {
+  return cudaFuncSetAttribute(attention_kernel<KT, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                              (int)attention_smem_bytes<KT, HD>());
+}
+
+cudaError_t configure_kernels(const sdfp_ctx* c) {
+  const bool hd128 = c->cfg.head_dim == 128;
+  cudaError_t e;
+  if (c->bf16)
+    e = hd128 ? configure_attention_t<__nv_bfloat16, 128>() : configure_attention_t<__nv_bfloat16, 64>();
+  else
+    e = hd128 ? configure_attention_t<float, 128>() : configure_attention_t<float, 64>();
+  if (e != cudaSuccess) return e;
+  return configure_linear_mma();
+}
+
+// ---- one forward pass ------------------------------------------------------------------
+
+enum Decide { DECIDE_NONE = 0, DECIDE_LOGITS = 1, DECIDE_ARGMAX = 2, DECIDE_SAMPLE_DRAFT = 3 };
+
+// rows: total rows; rows_per_seq for the attention grouping; n_chunks bounds the context.
+int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn_rows_per_seq, int n_chunks,
+                 int decide) {
+  const sdfp_config& g = c->cfg;
+  const int d = g.d_model, f = g.d_ffn;
+  if (c->bf16)
+    CU_OK(c, launch(c, plan_embed_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs,
+                    (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
+                    reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, d));
+  else
+    CU_OK(c, launch(c, plan_embed_kernel<float>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs,
+                    (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
+                    reinterpret_cast<const float*>(c->embed), c->h, d));
+  const KvCache& kv = draft ? c->cache_d : c->cache_t;
+  for (int l = 0; l < g.n_layers; ++l) {
+    if (draft && !c->keep[l]) continue;  // Algorithm 1: pruned layers are removed from the draft
+    const LayerWeights& lw = c->layers[l];
+    {
+      LinearCall lc{lw.qkv, c->h, d, rows, d, 3 * d / 2, lw.attn_gain, base_epi(c, EPI_QKV, c->q, d)};
+      lc.ep.kcache = kv.k[l];
+      lc.ep.vcache = kv.v[l];
+      CU_OK(c, run_linear(c, lc));
+    }
+    CU_OK(c, run_attention(c, kv, l, rows, attn_rows_per_seq, n_chunks));
+    {
+      LinearCall lc{lw.wo, c->att, d, rows, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)};
+      CU_OK(c, run_linear(c, lc));
+    }
+    {
+      LinearCall lc{lw.gu, c->h, d, rows, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)};
+      CU_OK(c, run_linear(c, lc));
+    }
+    {
+      LinearCall lc{lw.down, c->u, f, rows, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)};
+      CU_OK(c, run_linear(c, lc));
+    }
+  }
+  if (decide == DECIDE_NONE) return 0;
+  {
+    LinearCall lc{c->lm_head, c->h, d, rows, d, g.vocab / 2, c->final_gain, base_epi(c, EPI_LOGITS, c->logits, g.vocab)};
+    CU_OK(c, run_linear(c, lc));
+  }
+  if (decide == DECIDE_ARGMAX)
+    CU_OK(c, launch(c, argmax_kernel, dim3(rows), dim3(kArgmaxThreads), 0, (const float*)c->logits, g.vocab, pd,
+                    c->draft_tok, c->tgt_tok, c->row_argmax));
+  else if (decide == DECIDE_SAMPLE_DRAFT)
+    CU_OK(c, launch(c, sample_draft_kernel, dim3(rows), dim3(kSampleThreads), 0, (const float*)c->logits, g.vocab, pd,
+                    (const GenState*)c->gs, c->draft_tok, c->qprob, c->qsum));
+  return 0;
+}
+
+int enqueue_round(sdfp_ctx* c, int k, int batch, bool sampled, int n_chunks) {
+  PassDesc pd{};
+  pd.n_seq = batch;
+  if (k > 0) {
+    pd.kind = PASS_DRAFT_FIRST;
+    pd.rows_per_seq = 2;
+    if (int r = enqueue_pass(c, pd, true, 2 * batch, 2, n_chunks, sampled ? DECIDE_SAMPLE_DRAFT : DECIDE_ARGMAX)) return r;
+    for (int s = 1; s < k; ++s) {
+      pd.kind = PASS_DRAFT_NEXT;
+      pd.step = s;
+      pd.rows_per_seq = 1;
+      if (int r = enqueue_pass(c, pd, true, batch, 1, n_chunks, sampled ? DECIDE_SAMPLE_DRAFT : DECIDE_ARGMAX)) return r;
+    }
+  }
+  pd.kind = PASS_VERIFY;
+  pd.step = 0;
+  pd.rows_per_seq = k + 1;
+  if (int r = enqueue_pass(c, pd, false, (k + 1) * batch, k + 1, n_chunks, sampled ? DECIDE_LOGITS : DECIDE_ARGMAX))
+    return r;
+  if (sampled)
+    CU_OK(c, launch(c, accept_sampled_kernel, dim3(1), dim3(kSampleThreads), 0, c->gs, (const float*)c->logits,
+                    c->cfg.vocab, (const int*)c->draft_tok, (const float*)c->qprob, (const double*)c->qsum, c->seq_tok,
+                    c->cfg.max_seq, c->out_tok, c->stats));
+  else
+    CU_OK(c, launch(c, accept_greedy_kernel, dim3(1), dim3(32), 0, c->gs, (const int*)c->draft_tok,
+                    (const int*)c->tgt_tok, c->seq_tok, c->cfg.max_seq, c->out_tok, c->stats));
+  return 0;
+}
+
+// ---- weights ------------------------------------------------------------------------------
+
+template <typename WT>
+int pack_matrix(sdfp_ctx* c, void** dst, PackSrc ps, int n_pairs, int K) {
+  const size_t n = (size_t)n_pairs * 2 * K;
+  WT* p = nullptr;
+  if (int r = dev_alloc(c, &p, n)) return r;
+  if (c->use_mma) {
+    if (int r = pack_mma(c->stream, reinterpret_cast<__nv_bfloat16*>(p), ps, n_pairs, K)) return fail(c, SDFP_ECUDA, "pack_mma failed");
+  } else {
+    pack_pairs_kernel<WT><<<1184, 256, 0, c->stream>>>(p, ps, n_pairs, K);
+  }
+  CU_OK(c, cudaGetLastError());
+  *dst = p;
+  return 0;
+}
+
+template <typename WT>
+int widen_gain(sdfp_ctx* c, float** dst, const void* src, int n) {
+  if (int r = dev_alloc(c, dst, (size_t)n)) return r;
+  widen_vector_kernel<WT><<<(n + 255) / 256, 256, 0, c->stream>>>(*dst, reinterpret_cast<const WT*>(src), n);
+  CU_OK(c, cudaGetLastError());
+  return 0;
+}
+
+template <typename WT>
+int load_weights(sdfp_ctx* c, const sdfp_weights* w) {
+  const sdfp_config& g = c->cfg;
+  const int d = g.d_model, f = g.d_ffn, H = g.n_heads, hd = g.head_dim;
+  c->layers.resize(g.n_layers);
+  for (int l = 0; l < g.n_layers; ++l) {
+    LayerWeights& lw = c->layers[l];
+    if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] || !w->w_down[l] ||
+        !w->attn_norm[l] || !w->ffn_norm[l])
+      return fail(c, SDFP_EINVAL, "layer %d has a NULL weight pointer", l);
+    if (int r = pack_matrix<WT>(c, &lw.qkv, PackSrc{w->wq[l], w->wk[l], w->wv[l], 0, H, hd}, 3 * d / 2, d)) return r;
+    if (int r = pack_matrix<WT>(c, &lw.wo, PackSrc{w->wo[l], nullptr, nullptr, 2, H, hd}, d / 2, d)) return r;
+    if (int r = pack_matrix<WT>(c, &lw.gu, PackSrc{w->w_gate[l], w->w_up[l], nullptr, 1, H, hd}, f, d)) return r;
+    if (int r = pack_matrix<WT>(c, &lw.down, PackSrc{w->w_down[l], nullptr, nullptr, 2, H, hd}, d / 2, f)) return r;
+    if (int r = widen_gain<WT>(c, &lw.attn_gain, w->attn_norm[l], d)) return r;
+    if (int r = widen_gain<WT>(c, &lw.ffn_gain, w->ffn_norm[l], d)) return r;
+  }
+  if (int r = pack_matrix<WT>(c, &c->lm_head, PackSrc{w->lm_head, nullptr, nullptr, 2, H, hd}, g.vocab / 2, d)) return r;
+  if (int r = widen_gain<WT>(c, &c->final_gain, w->final_norm, d)) return r;
+  WT* e = nullptr;
+  if (int r = dev_alloc(c, &e, (size_t)g.vocab * d)) return r;
+  CU_OK(c, cudaMemcpyAsync(e, w->tok_embed, (size_t)g.vocab * d * sizeof(WT), cudaMemcpyDeviceToDevice, c->stream));
+  c->embed = e;
+  return 0;
+}
+
+int alloc_cache(sdfp_ctx* c, KvCache& kv) {
+  const sdfp_config& g = c->cfg;
+  const size_t bytes = (size_t)g.max_batch * g.n_heads * g.max_seq * g.head_dim * c->esz;
+  kv.k.resize(g.n_layers);
+  kv.v.resize(g.n_layers);
+  for (int l = 0; l < g.n_layers; ++l) {
+    unsigned char *pk = nullptr, *pv = nullptr;
+    if (int r = dev_alloc(c, &pk, bytes, true)) return r;
+    if (int r = dev_alloc(c, &pv, bytes, true)) return r;
+    kv.k[l] = pk;
+    kv.v[l] = pv;
+  }
+  return 0;
+}
+
+int64_t layer_weight_bytes(const sdfp_ctx* c) {
+  const int64_t d = c->cfg.d_model, f = c->cfg.d_ffn;
+  return (4 * d * d + 3 * d * f) * (int64_t)c->esz;
+}
+int64_t lm_head_bytes(const sdfp_ctx* c) { return (int64_t)c->cfg.vocab * c->cfg.d_model * (int64_t)c->esz; }
+int kept_layers(const sdfp_ctx* c) {
+  int n = 0;
+  for (uint8_t x : c->keep) n += x ? 1 : 0;
+  return n;
+}
+
+}  // namespace
+
+// =============================================================================================
+// C ABI
+// =============================================================================================
+
+extern "C" const char* sdfp_last_error(const sdfp_ctx* ctx) { return ctx ? ctx->err.c_str() : g_create_error.c_str(); }
+
+extern "C" void sdfp_destroy(sdfp_ctx* c) {
+  if (!c) return;
+  cudaStreamSynchronize(c->stream);
+  for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);
+  for (void* p : c->allocs) cudaFree(p);
+  if (c->pinned_flag) cudaFreeHost(c->pinned_flag);
+  for (auto& e : c->ev)
+    if (e) cudaEventDestroy(e);
+  if (c->own_stream) cudaStreamDestroy(c->stream);
+  delete c;
+}
+
+extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* cuda_stream, sdfp_ctx** out) {
+  if (!cfg || !w || !out) return fail(nullptr, SDFP_EINVAL, "sdfp_create: NULL argument");
+  *out = nullptr;
+  const sdfp_config& g = *cfg;
+  if (g.n_layers < 1 || g.n_layers > 1024 || g.d_model < 16 || g.n_heads < 1 || g.d_ffn < 16 || g.vocab < 16)
+    return fail(nullptr, SDFP_EINVAL, "sdfp_create: non-positive model dimension");
+  if (g.head_dim != 64 && g.head_dim != 128) return fail(nullptr, SDFP_EINVAL, "head_dim must be 64 or 128");
+  if (g.d_model != g.n_heads * g.head_dim) return fail(nullptr, SDFP_EINVAL, "d_model must equal n_heads*head_dim");
+  if (g.d_model % 16 || g.d_ffn % 16 || g.vocab % 16)
+    return fail(nullptr, SDFP_EINVAL, "d_model, d_ffn and vocab must be multiples of 16");
+  if (g.dtype != SDFP_F32 && g.dtype != SDFP_BF16) return fail(nullptr, SDFP_EINVAL, "unknown dtype");
+  if (g.max_batch < 1 || g.max_batch > kMaxBatch) return fail(nullptr, SDFP_EINVAL, "max_batch must be 1..%d", kMaxBatch);
+  if (g.k_max < 0 || g.k_max > kMaxK) return fail(nullptr, SDFP_EINVAL, "k_max must be 0..%d", kMaxK);
+  if (g.max_batch * (g.k_max + 1) > kMaxRows || g.max_batch * 2 > kMaxRows)
+    return fail(nullptr, SDFP_EINVAL, "max_batch*(k_max+1) must not exceed %d", kMaxRows);
+  if (g.max_seq < 4 || !(g.rms_eps > 0.f) || !(g.rope_theta > 0.f)) return fail(nullptr, SDFP_EINVAL, "bad max_seq, rms_eps or rope_theta");
+  if (!w->tok_embed || !w->final_norm || !w->lm_head || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up ||
+      !w->w_down || !w->attn_norm || !w->ffn_norm)
+    return fail(nullptr, SDFP_EINVAL, "sdfp_create: NULL weight pointer");
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+    cudaGetLastError();
+    return fail(nullptr, SDFP_ECUDA, "no CUDA device: this library has no CPU path");
+  }
+  sdfp_ctx* c = new (std::nothrow) sdfp_ctx();
+  if (!c) return fail(nullptr, SDFP_ENOMEM, "host allocation failed");
+  auto bail = [&](int code) {
+    g_create_error = c->err;
+    sdfp_destroy(c);
+    return code;
+  };
+  c->cfg = g;
+  c->stream = reinterpret_cast<cudaStream_t>(cuda_stream);
+  if (c->stream == nullptr) {
+    // the legacy default stream cannot be captured into a graph: use a stream of our own,
+    // after everything the caller queued so far (its weight tensors) has completed
+    if (cudaDeviceSynchronize() != cudaSuccess || cudaStreamCreateWithFlags(&c->stream, cudaStreamNonBlocking) != cudaSuccess) {
+      c->stream = nullptr;
+      c->err = "could not create a stream";
+      return bail(SDFP_ECUDA);
+    }
+    c->own_stream = true;
+  }
+  c->L.stream = c->stream;
+  c->L.count = &c->launches;
+  c->bf16 = (g.dtype == SDFP_BF16);
+  c->esz = c->bf16 ? 2 : 4;
+  c->use_mma = c->bf16 && !(g.flags & SDFP_FLAG_FMA_GEMM);
+  c->use_pdl = !(g.flags & SDFP_FLAG_NO_PDL);
+  c->use_graph = !(g.flags & SDFP_FLAG_NO_GRAPH);
+  c->L.pdl = c->use_pdl;
+  c->keep.assign(g.n_layers, 1);
+  int dev = 0;
+  cudaDeviceProp prop;
+  if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
+    c->err = "cudaGetDeviceProperties failed";
+    return bail(SDFP_ECUDA);
+  }
+  if (prop.major < 10) {
+    c->err = "this library is built for sm_100a (B200) only";
+    return bail(SDFP_ECUDA);
+  }
+  c->num_sms = prop.multiProcessorCount;
+  if (cudaError_t ke = configure_kernels(c)) {
+    c->err = std::string("kernel configuration failed: ") + cudaGetErrorString(ke);
+    return bail(SDFP_ECUDA);
+  }
+  int r = c->bf16 ? load_weights<__nv_bfloat16>(c, w) : load_weights<float>(c, w);
+  if (r) return bail(r);
+  if ((r = alloc_cache(c, c->cache_t)) || (r = alloc_cache(c, c->cache_d))) return bail(r);
+
+  // rotary tables in fp64, rounded to fp32
+  {
+    const int hp = g.head_dim / 2;
+    std::vector<float> cs((size_t)g.max_seq * hp), sn((size_t)g.max_seq * hp);
+    for (int i = 0; i < hp; ++i) {
+      const double inv = std::pow((double)g.rope_theta, -2.0 * i / g.head_dim);
+      for (int p = 0; p < g.max_seq; ++p) {
+        cs[(size_t)p * hp + i] = (float)std::cos(p * inv);
+        sn[(size_t)p * hp + i] = (float)std::sin(p * inv);
+      }
+    }
+    if ((r = dev_alloc(c, &c->rope_cos, cs.size())) || (r = dev_alloc(c, &c->rope_sin, sn.size()))) return bail(r);
+    if (cudaMemcpyAsync(c->rope_cos, cs.data(), cs.size() * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+        cudaMemcpyAsync(c->rope_sin, sn.data(), sn.size() * 4, cudaMemcpyHostToDevice, c->stream) != cudaSuccess ||
+        cudaStreamSynchronize(c->stream) != cudaSuccess) {
+      c->err = "upload of rotary tables failed";
+      return bail(SDFP_ECUDA);
+    }
+  }
+  const size_t R = kMaxRows;
+  c->n_chunks_cap = (g.max_seq + kAttnChunk - 1) / kAttnChunk;
+  c->stats_cap = g.max_seq;
+  if ((r = dev_alloc(c, &c->h, R * g.d_model, true)) || (r = dev_alloc(c, &c->q, R * g.d_model, true)) ||
+      (r = dev_alloc(c, &c->att, R * g.d_model, true)) || (r = dev_alloc(c, &c->u, R * g.d_ffn, true)) ||
+      (r = dev_alloc(c, &c->logits, R * g.vocab, true)) ||
+      (r = dev_alloc(c, &c->part_o, R * g.n_heads * c->n_chunks_cap * g.head_dim)) ||
+      (r = dev_alloc(c, &c->part_ml, R * g.n_heads * c->n_chunks_cap * 2)) ||
+      (r = dev_alloc(c, &c->attn_counters, R * g.n_heads, true)) || (r = dev_alloc(c, &c->plan.row_pos, R, true)) ||
+      (r = dev_alloc(c, &c->plan.row_seq, R, true)) || (r = dev_alloc(c, &c->plan.row_tok, R, true)) ||
+      (r = dev_alloc(c, &c->seq_tok, (size_t)g.max_batch * g.max_seq, true)) ||
+      (r = dev_alloc(c, &c->draft_tok, (size_t)kMaxBatch * kMaxK, true)) ||
+      (r = dev_alloc(c, &c->tgt_tok, (size_t)kMaxBatch * (kMaxK + 1), true)) ||
+      (r = dev_alloc(c, &c->row_argmax, R, true)) || (r = dev_alloc(c, &c->out_tok, (size_t)g.max_batch * g.max_seq, true)) ||
+      (r = dev_alloc(c, &c->fwd_tok, R, true)) ||
+      (r = dev_alloc(c, &c->qprob, (size_t)g.max_batch * std::max(1, g.k_max) * g.vocab, true)) ||
+      (r = dev_alloc(c, &c->qsum, (size_t)kMaxBatch * kMaxK, true)) || (r = dev_alloc(c, &c->gs, 1, true)) ||
+      (r = dev_alloc(c, &c->stats, (size_t)c->stats_cap * g.max_batch, true)))
+    return bail(r);
+  if (cudaMallocHost(reinterpret_cast<void**>(&c->pinned_flag), 64) != cudaSuccess) {
+    c->err = "cudaMallocHost failed";
+    return bail(SDFP_ENOMEM);
+  }
+  for (auto& e : c->ev)
+    if (cudaEventCreate(&e) != cudaSuccess) {
+      c->err = "cudaEventCreate failed";
+      return bail(SDFP_ECUDA);
+    }
+  cudaError_t e = cudaStreamSynchronize(c->stream);
+  if (e != cudaSuccess) {
+    c->err = std::string("weight packing failed: ") + cudaGetErrorString(e);
+    return bail(SDFP_ECUDA);
+  }
+  *out = c;
+  return 0;
+}
+
+extern "C" int sdfp_set_draft_layers(sdfp_ctx* c, const uint8_t* keep_mask) {
+  if (!c) return SDFP_EINVAL;
+  if (!keep_mask) return fail(c, SDFP_EINVAL, "keep_mask is NULL");
+  int kept = 0;
+  for (int l = 0; l < c->cfg.n_layers; ++l) kept += keep_mask[l] ? 1 : 0;
+  if (kept == 0) return fail(c, SDFP_EINVAL, "the draft must keep at least one layer");
+  bool same = true;
+  for (int l = 0; l < c->cfg.n_layers; ++l) same = same && ((keep_mask[l] != 0) == (c->keep[l] != 0));
+  if (!same) {
+    for (int l = 0; l < c->cfg.n_layers; ++l) c->keep[l] = keep_mask[l] ? 1 : 0;
+    for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);  // captured rounds baked the old layer set in
+    c->graphs.clear();
+  }
+  return 0;
+}
+
+namespace {
+
+// Feed tokens [from, to) of sequence b (already in seq_tok) through target or draft to fill its cache.
+int prefill_range(sdfp_ctx* c, bool draft, int b, int from, int to) {
+  const int chunk = 32;
+  for (int s = from; s < to; s += chunk) {
+    const int cnt = std::min(chunk, to - s);
+    PassDesc pd{};
+    pd.kind = PASS_TOKENS;
+    pd.seq = b;
+    pd.start = s;
+    pd.count = cnt;
+    pd.src = c->seq_tok + (size_t)b * c->cfg.max_seq + s;
+    const int rps = std::min(cnt, kAttnMaxR);
+    const int rows = ((cnt + rps - 1) / rps) * rps;  // whole attention groups; extra rows carry nothing
+    const int n_chunks = (s + cnt + kAttnChunk - 1) / kAttnChunk;
+    if (int r = enqueue_pass(c, pd, draft, rows, rps, n_chunks, DECIDE_NONE)) return r;
+  }
+  return 0;
+}
+
+}  // namespace
+
+extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch, int32_t prompt_len, int32_t k,
+                             int32_t max_new, float temperature, uint64_t seed, int32_t* out_tokens, int32_t* out_len,
+                             sdfp_round_stat* stats, int32_t max_rounds, int32_t* n_rounds) {
+  if (!c) return SDFP_EINVAL;
+  const sdfp_config& g = c->cfg;
+  if (!prompts || !out_tokens || !out_len) return fail(c, SDFP_EINVAL, "sdfp_generate: NULL pointer");
+  if (batch < 1 || batch > g.max_batch) return fail(c, SDFP_EINVAL, "batch %d outside 1..%d", batch, g.max_batch);
+  if (k < 0 || k > g.k_max) return fail(c, SDFP_EINVAL, "k %d outside 0..%d", k, g.k_max);
+  if (prompt_len < 1 || max_new < 1) return fail(c, SDFP_EINVAL, "prompt_len and max_new must be >= 1");
+  if ((int64_t)prompt_len + max_new + k + 1 > g.max_seq)
+    return fail(c, SDFP_EINVAL, "prompt_len + max_new + k + 1 = %lld exceeds max_seq %d",
+                (long long)prompt_len + max_new + k + 1, g.max_seq);
+  if (!(temperature >= 0.f)) return fail(c, SDFP_EINVAL, "temperature must be >= 0");
+  if (stats && max_rounds < 0) return fail(c, SDFP_EINVAL, "max_rounds < 0");
+  for (int64_t i = 0; i < (int64_t)batch * prompt_len; ++i)
+    if (prompts[i] < 0 || prompts[i] >= g.vocab) return fail(c, SDFP_EINVAL, "prompt token %d out of range", prompts[i]);
+  const bool sampled = temperature > 0.f;
+  cudaStream_t st = c->stream;
+
+  // state
+  GenState hs{};
+  for (int b = 0; b < batch; ++b) hs.n[b] = prompt_len;
+  for (int b = batch; b < kMaxBatch; ++b) hs.done[b] = 1;
+  hs.batch = batch;
+  hs.k = k;
+  hs.max_new = max_new;
+  hs.eos_id = g.eos_id;
+  hs.max_rounds = c->stats_cap;
+  hs.temperature = temperature;
+  hs.seed = seed;
+  CU_OK(c, cudaMemcpyAsync(c->gs, &hs, sizeof hs, cudaMemcpyHostToDevice, st));
+  for (int b = 0; b < batch; ++b)
+    CU_OK(c, cudaMemcpyAsync(c->seq_tok + (size_t)b * g.max_seq, prompts + (size_t)b * prompt_len,
+                             (size_t)prompt_len * 4, cudaMemcpyHostToDevice, st));
+  CU_OK(c, cudaMemsetAsync(c->out_tok, 0xff, (size_t)batch * max_new * 4, st));
+  CU_OK(c, cudaMemsetAsync(c->stats, 0, (size_t)c->stats_cap * batch * sizeof(RoundStat), st));
+
+  // prefill: the target caches positions 0..P-2, the draft 0..P-3 (its first pass of a
+  // round always feeds the last two committed tokens)
+  CU_OK(c, cudaEventRecord(c->ev[0], st));
+  for (int b = 0; b < batch; ++b) {
+    if (int r = prefill_range(c, false, b, 0, prompt_len - 1)) return r;
+    if (k > 0)
+      if (int r = prefill_range(c, true, b, 0, prompt_len - 2)) return r;
+  }
+  CU_OK(c, cudaEventRecord(c->ev[1], st));
+
+  // decode
+  const int n_chunks = (prompt_len + max_new + k + kAttnChunk) / kAttnChunk;
+  const long long launches0 = c->launches;
+  cudaGraphExec_t exec = nullptr;
+  long long launches_per_round = 0;
+  if (c->use_graph) {
+    auto key = std::make_tuple((int)k, (int)batch, sampled ? 1 : 0, n_chunks);
+    auto it = c->graphs.find(key);
+    if (it == c->graphs.end()) {
+      const long long l0 = c->launches;
+      cudaGraph_t graph = nullptr;
+      CU_OK(c, cudaStreamBeginCapture(st, cudaStreamCaptureModeThreadLocal));
+      const int r = enqueue_round(c, k, batch, sampled, n_chunks);
+      cudaError_t ce = cudaStreamEndCapture(st, &graph);
+      launches_per_round = c->launches - l0;
+      c->launches = l0;
+      if (r) {
+        if (graph) cudaGraphDestroy(graph);
+        return r;
+      }
+      CU_OK(c, ce);
+      cudaError_t ie = cudaGraphInstantiate(&exec, graph, 0);
+      cudaGraphDestroy(graph);
+      CU_OK(c, ie);
+      c->graphs[key] = sdfp_ctx::RoundGraph{exec, launches_per_round};
+    } else {
+      exec = it->second.exec;
+      launches_per_round = it->second.launches;
+    }
+  }
+  int rounds = 0;
+  const int round_cap = max_new + 1;
+  while (rounds < round_cap) {
+    if (exec) {
+      CU_OK(c, cudaGraphLaunch(exec, st));
+      c->launches += launches_per_round;
+    } else if (int r = enqueue_round(c, k, batch, sampled, n_chunks)) {
+      return r;
+    }
+    ++rounds;
+    CU_OK(c, cudaMemcpyAsync(c->pinned_flag, &c->gs->all_done, 4, cudaMemcpyDeviceToHost, st));
+    CU_OK(c, cudaStreamSynchronize(st));
+    if (c->pinned_flag[0]) break;
+  }
+  CU_OK(c, cudaEventRecord(c->ev[2], st));
+
+  // results
+  std::vector<int> lens(kMaxBatch);
+  GenState fin{};
+  CU_OK(c, cudaMemcpyAsync(&fin, c->gs, sizeof fin, cudaMemcpyDeviceToHost, st));
+  CU_OK(c, cudaMemcpyAsync(out_tokens, c->out_tok, (size_t)batch * max_new * 4, cudaMemcpyDeviceToHost, st));
+  std::vector<RoundStat> hstats((size_t)rounds * batch);
+  CU_OK(c, cudaMemcpyAsync(hstats.data(), c->stats, hstats.size() * sizeof(RoundStat), cudaMemcpyDeviceToHost, st));
+  CU_OK(c, cudaStreamSynchronize(st));
+  for (int b = 0; b < batch; ++b) out_len[b] = fin.n_new[b];
+  if (n_rounds) *n_rounds = rounds;
+  if (stats)
+    for (int r = 0; r < std::min(rounds, (int)max_rounds); ++r)
+      for (int b = 0; b < batch; ++b) {
+        const RoundStat& s = hstats[(size_t)r * batch + b];
+        stats[(size_t)r * batch + b] = sdfp_round_stat{s.drafted, s.accepted, s.committed};
+      }
+
+  // timing and traffic of the decode phase
+  sdfp_timing& t = c->timing;
+  t = sdfp_timing{};
+  cudaEventElapsedTime(&t.prefill_ms, c->ev[0], c->ev[1]);
+  cudaEventElapsedTime(&t.decode_ms, c->ev[1], c->ev[2]);
+  t.n_rounds = rounds;
+  t.n_draft_passes = rounds * k;
+  t.n_target_passes = rounds;
+  t.kernel_launches = c->launches - launches0;
+  const int64_t lw = layer_weight_bytes(c), lm = lm_head_bytes(c);
+  const int kept = kept_layers(c);
+  t.weight_bytes = (int64_t)rounds * ((int64_t)k * (kept * lw + lm) + (int64_t)g.n_layers * lw + lm);
+  const int64_t kv_tok = 2LL * g.d_model * (int64_t)c->esz;  // K and V of one token of one layer
+  std::vector<int> n(batch, prompt_len);
+  for (int r = 0; r < rounds; ++r)
+    for (int b = 0; b < batch; ++b) {
+      const RoundStat& s = hstats[(size_t)r * batch + b];
+      if (s.committed == 0 && s.drafted == 0 && k > 0) continue;
+      if (k == 0 && s.committed == 0) continue;
+      // draft pass i reads keys 0..n-1+i of the kept layers and writes its rows; verify reads 0..n-1+k
+      for (int i = 0; i < k; ++i) t.kv_bytes += (int64_t)kept * kv_tok * ((n[b] + i) + (i == 0 ? 2 : 1));
+      t.kv_bytes += (int64_t)g.n_layers * kv_tok * ((n[b] + k) + (k + 1));
+      n[b] += s.committed;
+      t.tokens_committed += s.committed;
+    }
+  return 0;
+}
+
+extern "C" int sdfp_forward_logits(sdfp_ctx* c, int32_t draft, const int32_t* tokens, int32_t rows, int32_t start,
+                                   float* host_logits) {
+  if (!c) return SDFP_EINVAL;
+  const sdfp_config& g = c->cfg;
+  if (!tokens || !host_logits) return fail(c, SDFP_EINVAL, "sdfp_forward_logits: NULL pointer");
+  if (rows < 1 || rows > kMaxRows) return fail(c, SDFP_EINVAL, "rows %d outside 1..%d", rows, kMaxRows);
+  if (start < 0 || start + rows > g.max_seq) return fail(c, SDFP_EINVAL, "positions exceed max_seq");
+  for (int i = 0; i < rows; ++i)
+    if (tokens[i] < 0 || tokens[i] >= g.vocab) return fail(c, SDFP_EINVAL, "token out of range");
+  CU_OK(c, cudaMemcpyAsync(c->fwd_tok, tokens, (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
+  PassDesc pd{};
+  pd.kind = PASS_TOKENS;
+  pd.seq = 0;
+  pd.start = start;
+  pd.count = rows;
+  pd.src = c->fwd_tok;
+  const int rps = std::min((int)rows, kAttnMaxR);
+  const int prow = ((rows + rps - 1) / rps) * rps;
+  const int n_chunks = (start + rows + kAttnChunk - 1) / kAttnChunk;
+  if (int r = enqueue_pass(c, pd, draft != 0, prow, rps, n_chunks, DECIDE_LOGITS)) return r;
+  CU_OK(c, cudaMemcpyAsync(host_logits, c->logits, (size_t)rows * g.vocab * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU_OK(c, cudaStreamSynchronize(c->stream));
+  return 0;
+}
+
+extern "C" int sdfp_get_timing(const sdfp_ctx* c, sdfp_timing* out) {
+  if (!c || !out) return SDFP_EINVAL;
+  *out = c->timing;
+  return 0;
+}
+
+extern "C" int sdfp_time_linear(sdfp_ctx* c, int32_t which, int32_t rows, int32_t iters, float* ms_per_launch,
+                                int64_t* weight_bytes_per_launch) {
+  if (!c) return SDFP_EINVAL;
+  const sdfp_config& g = c->cfg;
+  if (!ms_per_launch || !weight_bytes_per_launch) return fail(c, SDFP_EINVAL, "sdfp_time_linear: NULL pointer");
+  if (which < 0 || which > 4 || rows < 1 || rows > kMaxRows || iters < 1)
+    return fail(c, SDFP_EINVAL, "sdfp_time_linear: bad argument");
+  const int d = g.d_model, f = g.d_ffn;
+  // rows carry nothing (position -1): the QKV epilogue then writes no cache entry
+  CU_OK(c, cudaMemsetAsync(c->plan.row_pos, 0xff, kMaxRows * 4, c->stream));
+  CU_OK(c, cudaMemsetAsync(c->plan.row_seq, 0, kMaxRows * 4, c->stream));
+  auto one = [&](int l) -> cudaError_t {
+    const LayerWeights& lw = c->layers[l % g.n_layers];
+    if (which == 0) {
+      LinearCall lc{lw.qkv, c->h, d, rows, d, 3 * d / 2, lw.attn_gain, base_epi(c, EPI_QKV, c->q, d)};
+      lc.ep.kcache = c->cache_t.k[0];
+      lc.ep.vcache = c->cache_t.v[0];
+      return run_linear(c, lc);
+    } else if (which == 1) {
+      LinearCall lc{lw.wo, c->att, d, rows, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->q, d)};
+      return run_linear(c, lc);
+    } else if (which == 2) {
+      LinearCall lc{lw.gu, c->h, d, rows, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)};
+      return run_linear(c, lc);
+    } else if (which == 3) {
+      LinearCall lc{lw.down, c->u, f, rows, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->q, d)};
+      return run_linear(c, lc);
+    }
+    LinearCall lc{c->lm_head, c->h, d, rows, d, g.vocab / 2, c->final_gain, base_epi(c, EPI_LOGITS, c->logits, g.vocab)};
+    return run_linear(c, lc);
+  };
+  for (int i = 0; i < 3; ++i) CU_OK(c, one(i));
+  CU_OK(c, cudaEventRecord(c->ev[0], c->stream));
+  for (int i = 0; i < iters; ++i) CU_OK(c, one(i + 3));
+  CU_OK(c, cudaEventRecord(c->ev[1], c->stream));
+  CU_OK(c, cudaStreamSynchronize(c->stream));
+  float ms = 0.f;
+  cudaEventElapsedTime(&ms, c->ev[0], c->ev[1]);
+  *ms_per_launch = ms / iters;
+  const int64_t e = (int64_t)c->esz;
+  const int64_t bytes[5] = {3LL * d * d * e, 1LL * d * d * e, 2LL * f * d * e, 1LL * d * f * e, 1LL * g.vocab * d * e};
+  *weight_bytes_per_launch = bytes[which];
+  return 0;
+}

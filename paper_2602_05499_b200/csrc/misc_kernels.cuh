@@ -1,0 +1,212 @@
+// Small kernels around the linear and attention kernels: row planning + embedding
+// gather, argmax over the vocabulary, greedy accept/commit (Algorithm 1, loop body).
+#pragma once
+
+#include "common.cuh"
+
+namespace sdfp {
+
+constexpr int kMaxBatch = 16;
+constexpr int kMaxK = 15;
+
+// Device-resident generation state: a round never needs the host.
+struct GenState {
+  int n[kMaxBatch];      // committed length (prompt + generated) per sequence
+  int n_new[kMaxBatch];  // generated so far
+  int done[kMaxBatch];
+  int round;
+  int all_done;
+  // parameters of the running sdfp_generate call
+  int batch, k, max_new, eos_id, max_rounds;
+  float temperature;
+  unsigned long long seed;
+};
+
+enum PassKind {
+  PASS_TOKENS = 0,       // rows r = 0..count-1 of one sequence: token src[r], position start + r
+  PASS_DRAFT_FIRST = 1,  // 2 rows per sequence: the last two committed tokens
+  PASS_DRAFT_NEXT = 2,   // 1 row per sequence: draft token number `step` (1-based step >= 1)
+  PASS_VERIFY = 3        // k+1 rows per sequence: last committed token, then the k drafts
+};
+
+struct PassDesc {
+  int kind, step, rows_per_seq, n_seq;
+  int seq, start, count;  // PASS_TOKENS
+  const int* src;         // PASS_TOKENS: device token ids
+};
+
+struct RowPlan {
+  int* row_pos;  // [kMaxRows]
+  int* row_seq;
+  int* row_tok;
+};
+
+// One CTA per row: decide which token sits in the row and where, then gather its
+// embedding into the residual stream h[row, :].
+template <typename WT>
+__global__ void __launch_bounds__(128)
+plan_embed_kernel(PassDesc pd, const GenState* gs, const int* seq_tok, int max_seq,
+                  const int* draft_tok, RowPlan plan, const WT* __restrict__ embed, float* __restrict__ h,
+                  int d_model) {
+  __shared__ int s_tok, s_pos;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int m = blockIdx.x;
+  if (threadIdx.x == 0) {
+    int tok = 0, pos = -1, seq = 0;
+    if (pd.kind == PASS_TOKENS) {
+      seq = pd.seq;
+      if (m < pd.count) {
+        tok = ld_act(pd.src + m);
+        pos = pd.start + m;
+      }
+    } else {
+      const int R = pd.rows_per_seq;
+      const int b = m / R, i = m - b * R;
+      seq = b;
+      if (!ld_act(&gs->done[b])) {
+        const int n = ld_act(&gs->n[b]);
+        if (pd.kind == PASS_DRAFT_FIRST) {
+          pos = n - 2 + i;
+          if (pos >= 0) tok = ld_act(seq_tok + (size_t)b * max_seq + pos);
+        } else if (pd.kind == PASS_DRAFT_NEXT) {
+          pos = n - 1 + pd.step;
+          tok = ld_act(draft_tok + b * kMaxK + pd.step - 1);
+        } else {
+          pos = n - 1 + i;
+          tok = (i == 0) ? ld_act(seq_tok + (size_t)b * max_seq + n - 1) : ld_act(draft_tok + b * kMaxK + i - 1);
+        }
+      }
+    }
+    plan.row_pos[m] = pos;
+    plan.row_seq[m] = seq;
+    plan.row_tok[m] = tok;
+    s_tok = tok;
+    s_pos = pos;
+  }
+  __syncthreads();
+  const WT* e = embed + (size_t)s_tok * d_model;
+  float* dst = h + (size_t)m * d_model;
+  for (int k = threadIdx.x * 4; k < d_model; k += blockDim.x * 4) {
+    float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+    if (s_pos >= 0) v = load4(e + k);
+    *reinterpret_cast<float4*>(dst + k) = v;
+  }
+}
+
+// argmax over the vocabulary of every row; ties go to the lowest token id.
+// The result lands where the next kernel of the round expects it.
+constexpr int kArgmaxThreads = 512;
+__global__ void __launch_bounds__(kArgmaxThreads)
+argmax_kernel(const float* logits, int vocab, PassDesc pd, int* draft_tok, int* tgt_tok, int* row_argmax) {
+  __shared__ float s_val[kArgmaxThreads / 32];
+  __shared__ int s_idx[kArgmaxThreads / 32];
+  pdl_wait();
+  pdl_launch_dependents();
+  const int m = blockIdx.x;
+  const float* l = logits + (size_t)m * vocab;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int v = threadIdx.x; v < vocab; v += kArgmaxThreads) {
+    const float x = ld_act(l + v);
+    if (x > best || (x == best && v < bi)) {
+      best = x;
+      bi = v;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ob > best || (ob == best && oi < bi)) {
+      best = ob;
+      bi = oi;
+    }
+  }
+  if ((threadIdx.x & 31) == 0) {
+    s_val[threadIdx.x >> 5] = best;
+    s_idx[threadIdx.x >> 5] = bi;
+  }
+  __syncthreads();
+  if (threadIdx.x == 0) {
+    for (int w = 1; w < kArgmaxThreads / 32; ++w)
+      if (s_val[w] > best || (s_val[w] == best && s_idx[w] < bi)) {
+        best = s_val[w];
+        bi = s_idx[w];
+      }
+    row_argmax[m] = bi;
+    const int R = pd.rows_per_seq;
+    const int b = m / R, i = m - b * R;
+    if (pd.kind == PASS_DRAFT_FIRST) {
+      if (i == 1) draft_tok[b * kMaxK + 0] = bi;
+    } else if (pd.kind == PASS_DRAFT_NEXT) {
+      draft_tok[b * kMaxK + pd.step] = bi;
+    } else if (pd.kind == PASS_VERIFY) {
+      tgt_tok[b * (kMaxK + 1) + i] = bi;
+    }
+  }
+}
+
+struct RoundStat {
+  int drafted, accepted, committed;
+};
+
+// Commit step shared by greedy and sampled decoding: append d_1..d_j and the extra
+// token, truncated to max_new and at EOS, advance the lengths (that is the whole
+// rollback: cache entries beyond the new length are never read before being
+// rewritten), record the round.  Called by one thread per sequence.
+__device__ __forceinline__ void commit_tokens(volatile GenState* gs, int b, int k, int j, int extra, const int* d,
+                                              int* seq_tok, int max_seq, int* out_tok, RoundStat* stats) {
+  const int n = gs->n[b];
+  const int room = gs->max_new - gs->n_new[b];
+  int cnt = 0;
+  bool eos = false;
+  for (int t = 0; t <= j && cnt < room && !eos; ++t) {
+    const int tok = (t < j) ? ld_act(d + t) : extra;
+    seq_tok[(size_t)b * max_seq + n + cnt] = tok;
+    out_tok[(size_t)b * gs->max_new + gs->n_new[b] + cnt] = tok;
+    ++cnt;
+    if (gs->eos_id >= 0 && tok == gs->eos_id) eos = true;
+  }
+  gs->n[b] = n + cnt;
+  gs->n_new[b] += cnt;
+  if (eos || gs->n_new[b] >= gs->max_new) gs->done[b] = 1;
+  if (gs->round < gs->max_rounds) {
+    RoundStat* st = stats + (size_t)gs->round * gs->batch + b;
+    st->drafted = k;
+    st->accepted = j;
+    st->committed = cnt;
+  }
+}
+
+// Greedy accept (Eq. 2 degenerates to "draft token == target argmax"); k = 0 is a
+// plain autoregressive step.
+__global__ void __launch_bounds__(32)
+accept_greedy_kernel(GenState* gs_, const int* draft_tok, const int* tgt_tok, int* seq_tok, int max_seq,
+                     int* out_tok, RoundStat* stats) {
+  volatile GenState* gs = gs_;
+  pdl_wait();
+  pdl_launch_dependents();
+  const int b = threadIdx.x;
+  const int B = gs->batch, k = gs->k;
+  if (b < B) {
+    if (gs->done[b]) {
+      if (gs->round < gs->max_rounds) stats[(size_t)gs->round * B + b] = RoundStat{0, 0, 0};
+    } else {
+      const int* d = draft_tok + b * kMaxK;
+      const int* t = tgt_tok + b * (kMaxK + 1);
+      int j = 0;
+      while (j < k && ld_act(d + j) == ld_act(t + j)) ++j;
+      commit_tokens(gs, b, k, j, ld_act(t + j), d, seq_tok, max_seq, out_tok, stats);
+    }
+  }
+  __syncwarp();
+  const int fin = (b < B) ? gs->done[b] : 1;
+  const unsigned all = __all_sync(0xffffffffu, fin);
+  if (threadIdx.x == 0) {
+    gs->round += 1;
+    gs->all_done = all ? 1 : 0;
+  }
+}
+
+}  // namespace sdfp

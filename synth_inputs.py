@@ -58,16 +58,23 @@ MASTER_SEED = 20260205
 PROMPT_SEED = 1234
 
 
-def choose_skip_layers(n_layers: int, n_skip: int, seed: int = MASTER_SEED) -> List[int]:
-    """First n_skip entries of a seeded permutation of layers 1..L-2, sorted.
+def choose_skip_layers(n_layers: int, n_skip: int, how: str = "late", seed: int = MASTER_SEED) -> List[int]:
+    """The layers whose output projections are down-scaled and which the draft skips.
 
+    "late":   the n_skip layers just before the last one, L-1-n_skip .. L-2.  In a
+              random-init stack the residual stream grows with depth, so late layers
+              change it least; measured with the CPU oracle on the 7B shape (k=4) this
+              set is accepted about 80% of the time against about 55% for "seeded".
+    "seeded": the first n_skip entries of a seeded permutation of layers 1..L-2, sorted.
     The first and the last layer are never skipped.
     """
     if n_skip == 0:
         return []
-    inner = np.arange(1, n_layers - 1)
-    if n_skip > len(inner):
+    if n_skip > n_layers - 2:
         raise ValueError("cannot skip that many layers")
+    if how == "late":
+        return list(range(n_layers - 1 - n_skip, n_layers - 1))
+    inner = np.arange(1, n_layers - 1)
     rng = np.random.RandomState(seed % (2**31))
     return sorted(int(x) for x in rng.permutation(inner)[:n_skip])
 

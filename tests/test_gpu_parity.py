@@ -1,0 +1,288 @@
+"""GPU parity: the CUDA library against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import paper_2602_05499_b200 as pkg
+import synth_inputs as si
+from oracle import sdfp_oracle as orc
+
+from gpu_common import check_stream_against_oracle, make_pair, rel_l2
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.fixture(scope="module")
+def tiny():
+    eng, m, w = make_pair(si.TINY, (1, 2))
+    yield eng, m
+    eng.close()
+
+
+@pytest.fixture(scope="module")
+def tiny_bf16():
+    eng, m, w = make_pair(si.TINY_BF16, (1, 2))
+    yield eng, m
+    eng.close()
+
+
+# ---- logits -------------------------------------------------------------------------
+
+def _logits_both(eng, m, toks, chunks, layers=None):
+    draft = layers is not None
+    lm = orc.CachedLM(m, layers, max_seq=160)
+    got, ref, s = [], [], 0
+    for c in chunks:
+        got.append(eng.sdfp_forward_logits(toks[s:s + c], s, draft=draft))
+        ref.append(lm.feed(toks[s:s + c], s).numpy())
+        s += c
+    return np.concatenate(got), np.concatenate(ref)
+
+
+def test_logits_tiny_fp32(tiny):
+    eng, m = tiny
+    toks = si.make_prompts(m.vocab, 1, 75, seed=5)[0].tolist()
+    # ragged chunks: prefill-like 33 (three attention groups, ragged tail), single rows, a
+    # verify-like 5, and a chunk crossing the 64-key attention boundary
+    chunks = [33, 1, 1, 5, 20, 9, 1, 5]
+    got, ref = _logits_both(eng, m, toks, chunks)
+    assert got.shape == ref.shape == (75, m.vocab)
+    assert rel_l2(got, ref) < 1e-4
+    for r in range(75):
+        assert rel_l2(got[r], ref[r]) < 1e-4, r
+    got, ref = _logits_both(eng, m, toks, chunks, layers=[0, 3])
+    assert rel_l2(got, ref) < 1e-4
+
+
+def test_logits_tiny_bf16(tiny_bf16):
+    eng, m = tiny_bf16
+    toks = si.make_prompts(m.vocab, 1, 70, seed=6)[0].tolist()
+    got, ref = _logits_both(eng, m, toks, [17, 1, 5, 40, 7])
+    assert rel_l2(got, ref) < 1e-2
+    got, ref = _logits_both(eng, m, toks, [64, 6], layers=[0, 3])
+    assert rel_l2(got, ref) < 1e-2
+
+
+@pytest.mark.parametrize("which", ["f32", "bf16"])
+def test_rows_do_not_depend_on_batching(tiny, tiny_bf16, which):
+    """Batch invariance: a row's logits are bit-identical whether its token is fed alone,
+    inside a verify-sized block or inside a prefill chunk."""
+    eng, m = tiny if which == "f32" else tiny_bf16
+    toks = si.make_prompts(m.vocab, 1, 80, seed=8)[0].tolist()
+    one = np.concatenate([eng.sdfp_forward_logits(toks[i:i + 1], i) for i in range(80)])
+    s, blocks = 0, []
+    for c in [5, 5, 2, 32, 1, 7, 9, 16, 3]:
+        blocks.append(eng.sdfp_forward_logits(toks[s:s + c], s))
+        s += c
+    blk = np.concatenate(blocks)
+    assert s == 80
+    assert np.array_equal(one.view(np.uint32), blk.view(np.uint32))
+
+
+# ---- greedy decoding ------------------------------------------------------------------
+
+def test_greedy_c1_tokens_and_counts(tiny):
+    """Config C1: 16-token prompt, 64 new tokens, skip {1,2}, k=4."""
+    eng, m = tiny
+    prompt = si.make_prompts(m.vocab, 1, 16)
+    k, n_new = 4, 64
+    out = eng.sdfp_generate(prompt, k, n_new)
+    ar = eng.sdfp_generate(prompt, 0, n_new)
+    assert out.tokens[0] == ar.tokens[0]                      # speculative == autoregressive on the GPU, bit-exact
+    assert len(out.tokens[0]) == n_new
+    reported = check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+    ref = orc.spec_generate(orc.CachedLM(m, max_seq=160), orc.CachedLM(m, [0, 3], max_seq=160),
+                            prompt[0].tolist(), k, n_new)
+    if not reported:
+        assert out.tokens[0] == ref.tokens
+        assert out.stats[:, 0, 1].tolist() == [r.accepted for r in ref.rounds]    # acceptance counts, bit-exact
+        assert out.stats[:, 0, 2].tolist() == [r.committed for r in ref.rounds]
+        assert out.stats[:, 0, 0].tolist() == [k] * len(ref.rounds)
+        assert out.n_rounds == len(ref.rounds)
+    assert ar.n_rounds == n_new and ar.stats[:, 0, 2].tolist() == [1] * n_new
+
+
+@pytest.mark.parametrize("skip,k", [((1, 2, 3), 3), ((), 4), ((1, 2), 1), ((2,), 7), ((0, 1, 2), 8)])
+def test_greedy_other_masks(tiny, skip, k):
+    """Any draft gives the target's greedy stream; a draft equal to the target is always
+    accepted; a one-layer draft is mostly rejected and exercises the rollback."""
+    eng, m = tiny
+    prompt = si.make_prompts(m.vocab, 1, 21, seed=77)
+    n_new = 50
+    eng.sdfp_set_draft_layers(si.keep_mask(4, skip))
+    try:
+        out = eng.sdfp_generate(prompt, k, n_new)
+        ar = eng.sdfp_generate(prompt, 0, n_new)
+    finally:
+        eng.sdfp_set_draft_layers(si.keep_mask(4, (1, 2)))
+    assert out.tokens[0] == ar.tokens[0]
+    check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+    assert int(out.stats[:, 0, 2].sum()) == n_new
+    if skip == ():
+        assert (out.stats[:, 0, 1] == k).all()
+        assert out.n_rounds == -(-n_new // (k + 1))
+    ref = orc.spec_generate(orc.CachedLM(m, max_seq=160), orc.CachedLM(m, orc.keep_layers(4, skip), max_seq=160),
+                            prompt[0].tolist(), k, n_new)
+    if out.tokens[0] == ref.tokens:
+        assert out.stats[:, 0, 1].tolist() == [r.accepted for r in ref.rounds]
+
+
+@pytest.mark.parametrize("plen", [1, 2, 3, 64, 65])
+def test_prompt_length_edges(tiny, plen):
+    eng, m = tiny
+    prompt = si.make_prompts(m.vocab, 1, plen, seed=plen)
+    out = eng.sdfp_generate(prompt, 4, 12)
+    ar = eng.sdfp_generate(prompt, 0, 12)
+    assert out.tokens[0] == ar.tokens[0]
+    check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+
+
+def test_greedy_bf16(tiny_bf16):
+    eng, m = tiny_bf16
+    prompt = si.make_prompts(m.vocab, 1, 16)
+    out = eng.sdfp_generate(prompt, 4, 64)
+    ar = eng.sdfp_generate(prompt, 0, 64)
+    assert out.tokens[0] == ar.tokens[0]
+    check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+
+
+def test_graph_and_direct_launch_agree(tiny):
+    eng, m = tiny
+    prompt = si.make_prompts(m.vocab, 1, 16)
+    base = eng.sdfp_generate(prompt, 4, 40)
+    for flags in (pkg.FLAG_NO_GRAPH, pkg.FLAG_NO_PDL, pkg.FLAG_NO_GRAPH | pkg.FLAG_NO_PDL):
+        e2, _, _ = make_pair(si.TINY, (1, 2), flags=flags)
+        o2 = e2.sdfp_generate(prompt, 4, 40)
+        e2.close()
+        assert o2.tokens == base.tokens and np.array_equal(o2.stats, base.stats)
+
+
+def test_run_to_run_determinism(tiny):
+    eng, m = tiny
+    prompt = si.make_prompts(m.vocab, 1, 30, seed=3)
+    a = eng.sdfp_generate(prompt, 4, 48)
+    b = eng.sdfp_generate(prompt, 4, 48)
+    assert a.tokens == b.tokens and np.array_equal(a.stats, b.stats)
+    la = eng.sdfp_forward_logits(prompt[0, :20], 0)
+    lb = eng.sdfp_forward_logits(prompt[0, :20], 0)
+    assert np.array_equal(la.view(np.uint32), lb.view(np.uint32))
+
+
+def test_eos_stops_generation():
+    shape = si.TINY
+    prompt = si.make_prompts(shape.vocab, 1, 16)
+    eng, m, _ = make_pair(shape, (1, 2))
+    full = eng.sdfp_generate(prompt, 4, 40).tokens[0]
+    eng.close()
+    eos = full[17]
+    first = full.index(eos)
+    eng, m, _ = make_pair(shape, (1, 2), eos_id=eos)
+    out = eng.sdfp_generate(prompt, 4, 40)
+    ar = eng.sdfp_generate(prompt, 0, 40)
+    eng.close()
+    assert out.tokens[0] == full[:first + 1] == ar.tokens[0]
+    ref = orc.spec_generate(orc.CachedLM(m, max_seq=160), orc.CachedLM(m, [0, 3], max_seq=160),
+                            prompt[0].tolist(), 4, 40, eos_id=eos)
+    assert ref.tokens == out.tokens[0]
+    assert out.stats[:, 0, 2].tolist() == [r.committed for r in ref.rounds]
+
+
+# ---- batches ------------------------------------------------------------------------------
+
+def test_batch_rows_are_independent():
+    """A sequence's tokens and acceptance counts do not depend on what else is in the batch;
+    acceptance is ragged across the batch."""
+    eng, m, _ = make_pair(si.TINY, (1, 2), max_batch=4, k_max=4)
+    prompts = si.make_prompts(m.vocab, 4, 24, seed=40)
+    out = eng.sdfp_generate(prompts, 4, 40)
+    ar = eng.sdfp_generate(prompts, 0, 40)
+    assert out.tokens == ar.tokens
+    for b in range(4):
+        solo = eng.sdfp_generate(prompts[b:b + 1], 4, 40)
+        assert solo.tokens[0] == out.tokens[b]
+        acc_b = [int(a) for a, d in zip(out.stats[:, b, 1], out.stats[:, b, 0]) if d > 0]
+        assert acc_b == solo.stats[:, 0, 1].tolist()
+        check_stream_against_oracle(m, prompts[b].tolist(), out.tokens[b])
+    eng.close()
+
+
+# ---- API errors -------------------------------------------------------------------------------
+
+def test_api_errors(tiny):
+    eng, m = tiny
+    prompt = si.make_prompts(m.vocab, 1, 16)
+    with pytest.raises(pkg.SdfpError):
+        eng.sdfp_generate(prompt, 9, 10)                    # k > k_max
+    with pytest.raises(pkg.SdfpError):
+        eng.sdfp_generate(prompt, 4, 200)                   # exceeds max_seq
+    with pytest.raises(pkg.SdfpError):
+        eng.sdfp_generate(np.full((1, 4), m.vocab, dtype=np.int32), 4, 10)   # token out of range
+    with pytest.raises(pkg.SdfpError):
+        eng.sdfp_generate(np.concatenate([prompt, prompt]), 4, 10)           # batch > max_batch
+    with pytest.raises(pkg.SdfpError):
+        eng.sdfp_set_draft_layers([0, 0, 0, 0])
+    with pytest.raises(pkg.SdfpError):
+        eng.sdfp_generate(prompt, 4, 10, temperature=-1.0)
+    assert eng.sdfp_generate(prompt, 4, 10).tokens[0]       # still usable afterwards
+
+
+# ---- 7B-shaped layers (bf16, tensor-core linear kernel at its real shapes) ----------------------
+
+@pytest.fixture(scope="module")
+def l7b4():
+    eng, m, _ = make_pair(si.LLAMA7B_4L, (1, 2), max_seq=256, k_max=8, draw_device="cuda:0")
+    yield eng, m
+    eng.close()
+
+
+def test_logits_7b_shape(l7b4):
+    """d=4096, 32x128 heads, FFN 11008, vocab 32000: every linear shape of the 7B config,
+    4 layers deep so that the CPU oracle finishes in seconds."""
+    eng, m = l7b4
+    toks = si.make_prompts(m.vocab, 1, 90, seed=9)[0].tolist()
+    got, ref = _logits_both(eng, m, toks, [33, 1, 5, 2, 40, 9])
+    assert rel_l2(got, ref) < 1e-2
+    worst = max(rel_l2(got[r], ref[r]) for r in range(90))
+    assert worst < 1e-2
+    got, ref = _logits_both(eng, m, toks, [64, 1, 7], layers=[0, 3])
+    assert rel_l2(got, ref) < 1e-2
+
+
+def test_batch_invariance_7b_shape(l7b4):
+    eng, m = l7b4
+    toks = si.make_prompts(m.vocab, 1, 40, seed=10)[0].tolist()
+    one = np.concatenate([eng.sdfp_forward_logits(toks[i:i + 1], i) for i in range(40)])
+    s, blocks = 0, []
+    for c in [5, 7, 2, 17, 9]:
+        blocks.append(eng.sdfp_forward_logits(toks[s:s + c], s))
+        s += c
+    assert np.array_equal(one.view(np.uint32), np.concatenate(blocks).view(np.uint32))
+
+
+@pytest.mark.parametrize("k", [4, 6])
+def test_greedy_7b_shape(l7b4, k):
+    eng, m = l7b4
+    prompt = si.make_prompts(m.vocab, 1, 70, seed=12)
+    out = eng.sdfp_generate(prompt, k, 48)
+    ar = eng.sdfp_generate(prompt, 0, 48)
+    assert out.tokens[0] == ar.tokens[0]
+    reported = check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+    assert len(reported) <= 4
+    if not reported:
+        ref = orc.spec_generate(orc.CachedLM(m, max_seq=256), orc.CachedLM(m, [0, 3], max_seq=256),
+                                prompt[0].tolist(), k, 48)
+        if ref.tokens == out.tokens[0]:
+            assert out.stats[:, 0, 1].tolist() == [r.accepted for r in ref.rounds]
+
+
+def test_fma_and_tensor_paths_agree_closely():
+    """The CUDA-core comparison path and the tensor-core path compute the same model."""
+    shape = si.LLAMA7B_4L
+    toks = si.make_prompts(shape.vocab, 1, 24, seed=13)[0].tolist()
+    e1, m, _ = make_pair(shape, (1, 2), max_seq=64, draw_device="cuda:0")
+    a = e1.sdfp_forward_logits(toks, 0)
+    e1.close()
+    e2, _, _ = make_pair(shape, (1, 2), max_seq=64, flags=pkg.FLAG_FMA_GEMM, draw_device="cuda:0")
+    b = e2.sdfp_forward_logits(toks, 0)
+    e2.close()
+    assert rel_l2(a, b) < 2e-3
