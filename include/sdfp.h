@@ -159,6 +159,39 @@ int sdfp_generate(sdfp_ctx *ctx, const int32_t *prompts, int32_t batch, int32_t 
 int sdfp_forward_logits(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int32_t rows,
                         int32_t start, float *host_logits);
 
+/*
+ * sdfp_forward_logits without any allocation behind it.  (The paper has no counterpart:
+ * this is a packaging variant of the test hook above, not a step of the method.)
+ *
+ * Who needs it: code that is not allowed to reach a device allocator when it calls into the
+ * library.  Examples are a serving process whose own pool has claimed all of HBM, so that a
+ * later cudaMalloc fails or stalls the device; a real-time loop that must not take the
+ * implicit device-wide synchronisation cudaMalloc and cudaFree imply; and a thread that runs
+ * while another one captures a CUDA graph, during which allocation calls are illegal.  The
+ * split-KV attention kernel needs scratch in global memory (per (row, head, 64-key chunk) a
+ * partial max, sum and output vector, plus one arrival counter per head).  Here that scratch
+ * is a fixed array of SDFP_STATIC_SCRATCH_BYTES bytes compiled into the library, which every
+ * GPU that loads the library holds until the process exits.  The call uses no cudaMalloc,
+ * cudaFree, pool or framework allocator, directly or through another library.
+ *
+ * Arguments, results and errors are those of sdfp_forward_logits, and the logits are the same
+ * bit for bit.  In addition:
+ *   - SDFP_EINVAL when R x n_heads x ceil((start + rows) / 64) x (head_dim + 2) x 4 bytes,
+ *     plus the counters, exceed SDFP_STATIC_SCRATCH_BYTES, where R is the number of rows of
+ *     the widest pass the call runs (rows, rounded up to a multiple of 16 beyond 16).  The
+ *     message states both sizes.
+ *   - The first call on a device looks up the array's device address
+ *     (cudaGetSymbolAddress, with that device current) and keeps it.  Make that first call
+ *     before starting any stream capture.
+ *   - All contexts of the process on one device share the array, and it keeps what the last
+ *     call left in it.  The call clears the part that must start at zero itself, but two such
+ *     calls whose GPU work overlaps (different streams, different threads) race on it:
+ *     serialise them.
+ */
+#define SDFP_STATIC_SCRATCH_BYTES (8u << 20)
+int sdfp_forward_logits_static(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int32_t rows,
+                               int32_t start, float *host_logits);
+
 /* Timing of the last successful sdfp_generate. */
 int sdfp_get_timing(const sdfp_ctx *ctx, sdfp_timing *out);
 

@@ -16,7 +16,7 @@ SDFP_F32, SDFP_BF16 = 0, 1
 FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_FMA_GEMM = 1, 2, 4
 
 EXPORTS = ["sdfp_create", "sdfp_set_draft_layers", "sdfp_generate", "sdfp_forward_logits",
-           "sdfp_get_timing", "sdfp_time_linear", "sdfp_last_error", "sdfp_destroy"]
+           "sdfp_forward_logits_static", "sdfp_get_timing", "sdfp_time_linear", "sdfp_last_error", "sdfp_destroy"]
 
 
 class SdfpConfig(C.Structure):
@@ -77,6 +77,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdfp_forward_logits.argtypes = [vp, C.c_int32, C.POINTER(C.c_int32), C.c_int32, C.c_int32,
                                         C.POINTER(C.c_float)]
     lib.sdfp_forward_logits.restype = C.c_int
+    lib.sdfp_forward_logits_static.argtypes = lib.sdfp_forward_logits.argtypes
+    lib.sdfp_forward_logits_static.restype = C.c_int
     lib.sdfp_get_timing.argtypes = [vp, C.POINTER(SdfpTiming)]
     lib.sdfp_get_timing.restype = C.c_int
     lib.sdfp_time_linear.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_float),
@@ -193,6 +195,16 @@ class Sdfp:
         self._check(self.lib.sdfp_forward_logits(self.handle, 1 if draft else 0,
                                                  t.ctypes.data_as(C.POINTER(C.c_int32)), len(t), start,
                                                  out.ctypes.data_as(C.POINTER(C.c_float))))
+        return out
+
+    def sdfp_forward_logits_static(self, tokens: Sequence[int], start: int, draft: bool = False) -> np.ndarray:
+        """sdfp_forward_logits with the attention scratch in the library's static device array:
+        for callers that must not reach a device allocator.  Same arguments, same logits."""
+        t = np.ascontiguousarray(np.asarray(tokens, dtype=np.int32))
+        out = np.empty((len(t), self.shape.vocab), dtype=np.float32)
+        self._check(self.lib.sdfp_forward_logits_static(self.handle, 1 if draft else 0,
+                                                        t.ctypes.data_as(C.POINTER(C.c_int32)), len(t), start,
+                                                        out.ctypes.data_as(C.POINTER(C.c_float))))
         return out
 
     def sdfp_get_timing(self) -> Dict:

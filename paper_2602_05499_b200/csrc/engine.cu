@@ -730,6 +730,91 @@ extern "C" int sdfp_forward_logits(sdfp_ctx* c, int32_t draft, const int32_t* to
   return 0;
 }
 
+// ---- forward pass whose attention scratch is a static device array -----------------------------
+//
+// The split-KV attention kernel needs global scratch beyond its inputs and outputs: one
+// partial (max, sum, o[head_dim]) per (row, head, key chunk) and one arrival counter per
+// (sequence, head).  A context gets that scratch from cudaMalloc inside sdfp_create.  The
+// entry point below points the same kernel at a fixed array that is part of the library image
+// instead, so that the call itself reaches no allocator of any kind.
+namespace {
+
+constexpr size_t kStaticScratchBytes = SDFP_STATIC_SCRATCH_BYTES;
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+constexpr int kMaxDevices = 64;
+void* g_static_scratch_addr[kMaxDevices] = {};  // device address of the array, per device ordinal
+
+// In host code `g_static_scratch` is only a handle for the symbol; the address a kernel can
+// use has to be asked for, once per device, with that device current.
+int static_scratch_address(sdfp_ctx* c, unsigned char** out) {
+  int dev = -1;
+  CU_OK(c, cudaGetDevice(&dev));
+  if (dev < 0 || dev >= kMaxDevices) return fail(c, SDFP_ECUDA, "device ordinal %d not supported", dev);
+  if (!g_static_scratch_addr[dev]) {
+    void* p = nullptr;
+    CU_OK(c, cudaGetSymbolAddress(&p, g_static_scratch));
+    if (!p) return fail(c, SDFP_ECUDA, "cudaGetSymbolAddress returned a null address");
+    g_static_scratch_addr[dev] = p;
+  }
+  *out = reinterpret_cast<unsigned char*>(g_static_scratch_addr[dev]);
+  return 0;
+}
+
+size_t round_up_256(size_t n) { return (n + 255) & ~size_t(255); }
+
+}  // namespace
+
+extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int32_t* tokens, int32_t rows,
+                                          int32_t start, float* host_logits) {
+  if (!c) return SDFP_EINVAL;
+  const sdfp_config& g = c->cfg;
+  if (!tokens || !host_logits) return fail(c, SDFP_EINVAL, "sdfp_forward_logits_static: NULL pointer");
+  if (rows < 1 || rows > kMaxRows) return fail(c, SDFP_EINVAL, "rows %d outside 1..%d", rows, kMaxRows);
+  if (start < 0 || start + rows > g.max_seq) return fail(c, SDFP_EINVAL, "positions exceed max_seq");
+  for (int i = 0; i < rows; ++i)
+    if (tokens[i] < 0 || tokens[i] >= g.vocab) return fail(c, SDFP_EINVAL, "token out of range");
+  const int rps = std::min((int)rows, kAttnMaxR);
+  const int prow = ((rows + rps - 1) / rps) * rps;
+  const int n_chunks = (start + rows + kAttnChunk - 1) / kAttnChunk;
+  // layout inside the array: arrival counters | (max, sum) partials | o partials
+  const size_t counters_bytes = round_up_256((size_t)kMaxRows * g.n_heads * sizeof(int));
+  const size_t ml_bytes = round_up_256((size_t)prow * g.n_heads * n_chunks * 2 * sizeof(float));
+  const size_t o_bytes = round_up_256((size_t)prow * g.n_heads * n_chunks * g.head_dim * sizeof(float));
+  const size_t need = counters_bytes + ml_bytes + o_bytes;
+  if (need > kStaticScratchBytes)
+    return fail(c, SDFP_EINVAL,
+                "sdfp_forward_logits_static: %d rows x %d heads x %d key chunks need %zu bytes of attention scratch, "
+                "the static array holds %zu; use fewer rows per call, a shorter context, or sdfp_forward_logits",
+                prow, g.n_heads, n_chunks, need, kStaticScratchBytes);
+  unsigned char* base = nullptr;
+  if (int r = static_scratch_address(c, &base)) return r;
+  // the array keeps whatever the previous call (of any context) left: the counters must start at zero
+  CU_OK(c, cudaMemsetAsync(base, 0, counters_bytes, c->stream));
+  CU_OK(c, cudaMemcpyAsync(c->fwd_tok, tokens, (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
+  PassDesc pd{};
+  pd.kind = PASS_TOKENS;
+  pd.seq = 0;
+  pd.start = start;
+  pd.count = rows;
+  pd.src = c->fwd_tok;
+  // same pass as sdfp_forward_logits, with the attention scratch pointers swapped for its duration
+  float* const own_o = c->part_o;
+  float* const own_ml = c->part_ml;
+  int* const own_counters = c->attn_counters;
+  c->attn_counters = reinterpret_cast<int*>(base);
+  c->part_ml = reinterpret_cast<float*>(base + counters_bytes);
+  c->part_o = reinterpret_cast<float*>(base + counters_bytes + ml_bytes);
+  const int r = enqueue_pass(c, pd, draft != 0, prow, rps, n_chunks, DECIDE_LOGITS);
+  c->part_o = own_o;
+  c->part_ml = own_ml;
+  c->attn_counters = own_counters;
+  if (r) return r;
+  CU_OK(c, cudaMemcpyAsync(host_logits, c->logits, (size_t)rows * g.vocab * 4, cudaMemcpyDeviceToHost, c->stream));
+  CU_OK(c, cudaStreamSynchronize(c->stream));
+  return 0;
+}
+
 extern "C" int sdfp_get_timing(const sdfp_ctx* c, sdfp_timing* out) {
   if (!c || !out) return SDFP_EINVAL;
   *out = c->timing;
