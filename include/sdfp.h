@@ -49,6 +49,8 @@ typedef enum { SDFP_F32 = 0, SDFP_BF16 = 1 } sdfp_dtype;
 #define SDFP_FLAG_NO_GRAPH 1u /* launch kernels directly instead of replaying CUDA graphs    */
 #define SDFP_FLAG_NO_PDL 2u   /* no programmatic dependent launch between consecutive kernels */
 #define SDFP_FLAG_FMA_GEMM 4u /* bf16 models: CUDA-core FMA GEMM instead of the tensor path  */
+#define SDFP_FLAG_NO_PASS_KERNEL 8u /* bf16 models: one kernel per operation instead of the
+                                       persistent whole-pass kernel                            */
 
 /*
  * Model and capacity description.  The decoder is the LLaMA-2 architecture the
@@ -178,8 +180,9 @@ int sdfp_forward_logits(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int
  * bit for bit.  In addition:
  *   - SDFP_EINVAL when R x n_heads x ceil((start + rows) / 64) x (head_dim + 2) x 4 bytes,
  *     plus the counters, exceed SDFP_STATIC_SCRATCH_BYTES, where R is the number of rows of
- *     the widest pass the call runs (rows, rounded up to a multiple of 16 beyond 16).  The
- *     message states both sizes.
+ *     the widest pass the call runs (rows, but at most 16 for bf16 models, which are served
+ *     in passes of 16 rows; rounded up to a multiple of 16 beyond 16).  The message states
+ *     both sizes.
  *   - The first call on a device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and keeps it.  Make that first call
  *     before starting any stream capture.

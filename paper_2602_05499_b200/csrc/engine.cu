@@ -26,6 +26,7 @@
 #include "linear_fma.cuh"
 #include "linear_mma.cuh"
 #include "misc_kernels.cuh"
+#include "pass_kernel.cuh"
 #include "sampling.cuh"
 
 using namespace sdfp;
@@ -88,6 +89,17 @@ struct sdfp_ctx {
   std::map<std::tuple<int, int, int, int>, RoundGraph> graphs;  // (k, batch, sampled, n_chunks)
   long long launches = 0;
   Launcher L{};
+
+  // persistent pass kernel (bf16 tensor path, passes of up to kPassMaxRows rows)
+  bool use_pass = false;
+  StageDesc *prog_t = nullptr, *prog_d = nullptr;  // device: stage lists of the target and of the draft
+  int n_prog_t = 0, n_prog_d = 0;
+  PassSync* psync = nullptr;
+  float* split_partials = nullptr;
+  unsigned* split_flags = nullptr;
+  int pass_slots = 0;
+  size_t pass_smem = 0;
+  int pass_grid = 0;
   bool own_stream = false;
   sdfp_timing timing{};
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
@@ -220,6 +232,127 @@ cudaError_t configure_kernels(const sdfp_ctx* c) {
   return configure_linear_mma();
 }
 
+// ---- persistent pass kernel: stage lists and launch ---------------------------------------------
+
+StageDesc linear_desc(const void* w, const float* x, int K, int n_pairs, const float* gain, const EpiParams& ep) {
+  StageDesc s{};
+  s.kind = ST_LINEAR;
+  s.K = K;
+  s.KT = K / 16;
+  s.NT = n_pairs / 8;
+  s.n_groups = (s.NT + kUnitTiles - 1) / kUnitTiles;
+  s.ldx = K;
+  s.W = reinterpret_cast<const uint4*>(w);
+  s.X = x;
+  s.gain = gain;
+  s.ep = ep;
+  return s;
+}
+
+// The stage list of one forward pass: the target runs every layer, the draft the kept ones
+// (Algorithm 1: the draft is the model with the pruned layers removed).  The lm-head is the
+// last stage, so a pass that needs no logits runs the list without its last entry.
+int build_program(sdfp_ctx* c, bool draft, StageDesc** dev, int* n_out) {
+  const sdfp_config& g = c->cfg;
+  const int d = g.d_model, f = g.d_ffn;
+  const KvCache& kv = draft ? c->cache_d : c->cache_t;
+  std::vector<StageDesc> prog;
+  for (int l = 0; l < g.n_layers; ++l) {
+    if (draft && !c->keep[l]) continue;
+    const LayerWeights& lw = c->layers[l];
+    EpiParams qkv = base_epi(c, EPI_QKV, c->q, d);
+    qkv.kcache = kv.k[l];
+    qkv.vcache = kv.v[l];
+    prog.push_back(linear_desc(lw.qkv, c->h, d, 3 * d / 2, lw.attn_gain, qkv));
+    StageDesc at{};
+    at.kind = ST_ATTN;
+    at.X = c->q;
+    at.ep = base_epi(c, EPI_RESID, c->att, d);
+    at.ep.kcache = kv.k[l];
+    at.ep.vcache = kv.v[l];
+    prog.push_back(at);
+    prog.push_back(linear_desc(lw.wo, c->att, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+    prog.push_back(linear_desc(lw.gu, c->h, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
+    prog.push_back(linear_desc(lw.down, c->u, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+  }
+  prog.push_back(linear_desc(c->lm_head, c->h, d, g.vocab / 2, c->final_gain, base_epi(c, EPI_LOGITS, c->logits, g.vocab)));
+  if (*dev == nullptr)
+    if (int r = dev_alloc(c, dev, (size_t)5 * g.n_layers + 1)) return r;
+  CU_OK(c, cudaMemcpyAsync(*dev, prog.data(), prog.size() * sizeof(StageDesc), cudaMemcpyHostToDevice, c->stream));
+  CU_OK(c, cudaStreamSynchronize(c->stream));  // prog is a local
+  *n_out = (int)prog.size();
+  return 0;
+}
+
+int build_programs(sdfp_ctx* c) {
+  if (!c->use_pass) return 0;
+  if (int r = build_program(c, false, &c->prog_t, &c->n_prog_t)) return r;
+  return build_program(c, true, &c->prog_d, &c->n_prog_d);
+}
+
+template <int CG, int HD>
+size_t pass_smem_bytes(int n_slots) {
+  return (size_t)n_slots * kSlotBytes + pass_work_bytes<CG, HD>() + sizeof(PassShared);
+}
+
+// Largest ring that fits beside the work area of the widest instantiation (two column groups).
+template <int HD>
+cudaError_t configure_pass_t(sdfp_ctx* c, int max_smem_optin) {
+  int n_slots = 16;
+  while (n_slots > 2 && pass_smem_bytes<2, HD>(n_slots) > (size_t)max_smem_optin) --n_slots;
+  c->pass_slots = n_slots;
+  c->pass_smem = pass_smem_bytes<2, HD>(n_slots);
+  cudaError_t e = cudaFuncSetAttribute(pass_kernel<1, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_smem);
+  if (e != cudaSuccess) return e;
+  e = cudaFuncSetAttribute(pass_kernel<2, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_smem);
+  if (e != cudaSuccess) return e;
+  // a cooperative launch needs every CTA resident at once: one per SM
+  int per_sm = 0;
+  e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pass_kernel<2, HD>, kPassThreads, c->pass_smem);
+  if (e != cudaSuccess) return e;
+  if (per_sm < 1) return cudaErrorLaunchOutOfResources;
+  c->pass_grid = c->num_sms;
+  return cudaSuccess;
+}
+
+template <int CG, int HD>
+cudaError_t launch_pass_t(sdfp_ctx* c, const PassParams& pp) {
+  cudaLaunchConfig_t lc = {};
+  lc.gridDim = dim3(c->pass_grid);
+  lc.blockDim = dim3(kPassThreads);
+  lc.dynamicSmemBytes = c->pass_smem;
+  lc.stream = c->stream;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeCooperative;
+  attr[0].val.cooperative = 1;
+  lc.attrs = attr;
+  lc.numAttrs = 1;
+  c->launches += 1;
+  return cudaLaunchKernelEx(&lc, pass_kernel<CG, HD>, pp, c->pass_slots);
+}
+
+cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, int n_chunks, bool with_lm_head) {
+  PassParams pp{};
+  pp.prog = draft ? c->prog_d : c->prog_t;
+  pp.n_stages = (draft ? c->n_prog_d : c->n_prog_t) - (with_lm_head ? 0 : 1);
+  pp.M = rows;
+  pp.rows_per_seq = rows_per_seq;
+  pp.n_chunks = n_chunks;
+  pp.row_pos = c->plan.row_pos;
+  pp.row_seq = c->plan.row_seq;
+  pp.eps = c->cfg.rms_eps;
+  pp.attn_scale = 1.0f / std::sqrt((float)c->cfg.head_dim);
+  pp.part_o = c->part_o;
+  pp.part_ml = c->part_ml;
+  pp.attn_counters = c->attn_counters;
+  pp.split_partials = c->split_partials;
+  pp.split_flags = c->split_flags;
+  pp.sync = c->psync;
+  const bool hd128 = c->cfg.head_dim == 128;
+  if (rows <= 8) return hd128 ? launch_pass_t<1, 128>(c, pp) : launch_pass_t<1, 64>(c, pp);
+  return hd128 ? launch_pass_t<2, 128>(c, pp) : launch_pass_t<2, 64>(c, pp);
+}
+
 // ---- one forward pass ------------------------------------------------------------------
 
 enum Decide { DECIDE_NONE = 0, DECIDE_LOGITS = 1, DECIDE_ARGMAX = 2, DECIDE_SAMPLE_DRAFT = 3 };
@@ -238,7 +371,9 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
                     (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
                     reinterpret_cast<const float*>(c->embed), c->h, d));
   const KvCache& kv = draft ? c->cache_d : c->cache_t;
-  for (int l = 0; l < g.n_layers; ++l) {
+  const bool whole_pass = c->use_pass && rows <= kPassMaxRows;
+  if (whole_pass) CU_OK(c, run_pass(c, draft, rows, attn_rows_per_seq, n_chunks, decide != DECIDE_NONE));
+  for (int l = 0; l < g.n_layers && !whole_pass; ++l) {
     if (draft && !c->keep[l]) continue;  // Algorithm 1: pruned layers are removed from the draft
     const LayerWeights& lw = c->layers[l];
     {
@@ -262,7 +397,7 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
     }
   }
   if (decide == DECIDE_NONE) return 0;
-  {
+  if (!whole_pass) {
     LinearCall lc{c->lm_head, c->h, d, rows, d, g.vocab / 2, c->final_gain, base_epi(c, EPI_LOGITS, c->logits, g.vocab)};
     CU_OK(c, run_linear(c, lc));
   }
@@ -308,11 +443,12 @@ int enqueue_round(sdfp_ctx* c, int k, int batch, bool sampled, int n_chunks) {
 
 template <typename WT>
 int pack_matrix(sdfp_ctx* c, void** dst, PackSrc ps, int n_pairs, int K) {
-  const size_t n = (size_t)n_pairs * 2 * K;
+  const int n_groups = (n_pairs / 8 + kUnitTiles - 1) / kUnitTiles;
+  const size_t n = c->use_mma ? (size_t)n_groups * (K / 16) * (kUnitBytes / 2) : (size_t)n_pairs * 2 * K;
   WT* p = nullptr;
   if (int r = dev_alloc(c, &p, n)) return r;
   if (c->use_mma) {
-    if (int r = pack_mma(c->stream, reinterpret_cast<__nv_bfloat16*>(p), ps, n_pairs, K)) return fail(c, SDFP_ECUDA, "pack_mma failed");
+    pack_units_kernel<<<1184, 256, 0, c->stream>>>(reinterpret_cast<__nv_bfloat16*>(p), ps, n_pairs, K, n_groups);
   } else {
     pack_pairs_kernel<WT><<<1184, 256, 0, c->stream>>>(p, ps, n_pairs, K);
   }
@@ -464,6 +600,16 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
     return bail(SDFP_ECUDA);
   }
   c->num_sms = prop.multiProcessorCount;
+  c->use_pass = c->use_mma && !(g.flags & SDFP_FLAG_NO_PASS_KERNEL) && prop.cooperativeLaunch && g.d_model >= 64;
+  if (c->use_pass) {
+    int optin = 0;
+    cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+    const cudaError_t pe = g.head_dim == 128 ? configure_pass_t<128>(c, optin) : configure_pass_t<64>(c, optin);
+    if (pe != cudaSuccess) {
+      c->err = std::string("pass kernel configuration failed: ") + cudaGetErrorString(pe);
+      return bail(SDFP_ECUDA);
+    }
+  }
   if (cudaError_t ke = configure_kernels(c)) {
     c->err = std::string("kernel configuration failed: ") + cudaGetErrorString(ke);
     return bail(SDFP_ECUDA);
@@ -510,6 +656,12 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
       (r = dev_alloc(c, &c->qsum, (size_t)kMaxBatch * kMaxK, true)) || (r = dev_alloc(c, &c->gs, 1, true)) ||
       (r = dev_alloc(c, &c->stats, (size_t)c->stats_cap * g.max_batch, true)))
     return bail(r);
+  if (c->use_pass) {
+    if ((r = dev_alloc(c, &c->psync, 1, true)) ||
+        (r = dev_alloc(c, &c->split_partials, (size_t)c->pass_grid * kUnitTiles * 2 * 64 * 2, true)) ||
+        (r = dev_alloc(c, &c->split_flags, (size_t)c->pass_grid, true)) || (r = build_programs(c)))
+      return bail(r);
+  }
   if (cudaMallocHost(reinterpret_cast<void**>(&c->pinned_flag), 64) != cudaSuccess) {
     c->err = "cudaMallocHost failed";
     return bail(SDFP_ENOMEM);
@@ -540,15 +692,64 @@ extern "C" int sdfp_set_draft_layers(sdfp_ctx* c, const uint8_t* keep_mask) {
     for (int l = 0; l < c->cfg.n_layers; ++l) c->keep[l] = keep_mask[l] ? 1 : 0;
     for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);  // captured rounds baked the old layer set in
     c->graphs.clear();
+    CU_OK(c, cudaStreamSynchronize(c->stream));
+    if (int r = build_programs(c)) return r;
   }
   return 0;
 }
 
 namespace {
 
+// A failed wait inside the pass kernel leaves its code in device memory; turn it into an error
+// and put the synchronisation words back to their initial state.
+int check_pass_error(sdfp_ctx* c) {
+  if (!c->use_pass) return 0;
+  PassSync ps{};
+  CU_OK(c, cudaMemcpyAsync(&ps, c->psync, sizeof ps, cudaMemcpyDeviceToHost, c->stream));
+  CU_OK(c, cudaStreamSynchronize(c->stream));
+  if (ps.error == 0) return 0;
+  cudaMemsetAsync(c->psync, 0, sizeof(PassSync), c->stream);
+  cudaMemsetAsync(c->split_flags, 0, (size_t)c->pass_grid * sizeof(unsigned), c->stream);
+  cudaMemsetAsync(c->attn_counters, 0, (size_t)kMaxRows * c->cfg.n_heads * sizeof(int), c->stream);
+  cudaStreamSynchronize(c->stream);
+  static const char* const what[] = {"", "grid barrier", "weight slot never filled", "weight slot never freed",
+                                     "partial sum of a split group never posted"};
+  return fail(c, SDFP_ECUDA, "pass kernel gave up a wait (%s); results of this call are invalid",
+              ps.error >= 1 && ps.error <= 4 ? what[ps.error] : "unknown");
+}
+
+// Logits of `rows` tokens of sequence slot 0 at positions start.., in passes of as many rows as
+// one pass carries, so that a row's logits never depend on how many rows the caller asked for.
+int forward_logits_passes(sdfp_ctx* c, bool draft, const int32_t* tokens, int rows, int start, float* host_logits) {
+  const sdfp_config& g = c->cfg;
+  CU_OK(c, cudaMemcpyAsync(c->fwd_tok, tokens, (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
+  const int per_pass = c->use_pass ? kPassMaxRows : kMaxRows;
+  for (int off = 0; off < rows; off += per_pass) {
+    const int cnt = std::min(per_pass, rows - off);
+    PassDesc pd{};
+    pd.kind = PASS_TOKENS;
+    pd.seq = 0;
+    pd.start = start + off;
+    pd.count = cnt;
+    pd.src = c->fwd_tok + off;
+    const int rps = std::min(cnt, kAttnMaxR);
+    const int prow = ((cnt + rps - 1) / rps) * rps;
+    const int n_chunks = (start + off + cnt + kAttnChunk - 1) / kAttnChunk;
+    if (int r = enqueue_pass(c, pd, draft, prow, rps, n_chunks, DECIDE_LOGITS)) return r;
+    CU_OK(c, cudaMemcpyAsync(host_logits + (size_t)off * g.vocab, c->logits, (size_t)cnt * g.vocab * 4,
+                             cudaMemcpyDeviceToHost, c->stream));
+  }
+  CU_OK(c, cudaStreamSynchronize(c->stream));
+  return check_pass_error(c);
+}
+
+}  // namespace
+
+namespace {
+
 // Feed tokens [from, to) of sequence b (already in seq_tok) through target or draft to fill its cache.
 int prefill_range(sdfp_ctx* c, bool draft, int b, int from, int to) {
-  const int chunk = 32;
+  const int chunk = c->use_pass ? kPassMaxRows : 32;
   for (int s = from; s < to; s += chunk) {
     const int cnt = std::min(chunk, to - s);
     PassDesc pd{};
@@ -659,6 +860,7 @@ extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch,
     if (c->pinned_flag[0]) break;
   }
   CU_OK(c, cudaEventRecord(c->ev[2], st));
+  if (int r = check_pass_error(c)) return r;
 
   // results
   std::vector<int> lens(kMaxBatch);
@@ -714,20 +916,7 @@ extern "C" int sdfp_forward_logits(sdfp_ctx* c, int32_t draft, const int32_t* to
   if (start < 0 || start + rows > g.max_seq) return fail(c, SDFP_EINVAL, "positions exceed max_seq");
   for (int i = 0; i < rows; ++i)
     if (tokens[i] < 0 || tokens[i] >= g.vocab) return fail(c, SDFP_EINVAL, "token out of range");
-  CU_OK(c, cudaMemcpyAsync(c->fwd_tok, tokens, (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
-  PassDesc pd{};
-  pd.kind = PASS_TOKENS;
-  pd.seq = 0;
-  pd.start = start;
-  pd.count = rows;
-  pd.src = c->fwd_tok;
-  const int rps = std::min((int)rows, kAttnMaxR);
-  const int prow = ((rows + rps - 1) / rps) * rps;
-  const int n_chunks = (start + rows + kAttnChunk - 1) / kAttnChunk;
-  if (int r = enqueue_pass(c, pd, draft != 0, prow, rps, n_chunks, DECIDE_LOGITS)) return r;
-  CU_OK(c, cudaMemcpyAsync(host_logits, c->logits, (size_t)rows * g.vocab * 4, cudaMemcpyDeviceToHost, c->stream));
-  CU_OK(c, cudaStreamSynchronize(c->stream));
-  return 0;
+  return forward_logits_passes(c, draft != 0, tokens, rows, start, host_logits);
 }
 
 // ---- forward pass whose attention scratch is a static device array -----------------------------
@@ -774,8 +963,10 @@ extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int3
   if (start < 0 || start + rows > g.max_seq) return fail(c, SDFP_EINVAL, "positions exceed max_seq");
   for (int i = 0; i < rows; ++i)
     if (tokens[i] < 0 || tokens[i] >= g.vocab) return fail(c, SDFP_EINVAL, "token out of range");
-  const int rps = std::min((int)rows, kAttnMaxR);
-  const int prow = ((rows + rps - 1) / rps) * rps;
+  // the widest pass this call will run, and the longest context any of its passes sees
+  const int per_pass = std::min((int)rows, c->use_pass ? kPassMaxRows : kMaxRows);
+  const int rps = std::min(per_pass, kAttnMaxR);
+  const int prow = ((per_pass + rps - 1) / rps) * rps;
   const int n_chunks = (start + rows + kAttnChunk - 1) / kAttnChunk;
   // layout inside the array: arrival counters | (max, sum) partials | o partials
   const size_t counters_bytes = round_up_256((size_t)kMaxRows * g.n_heads * sizeof(int));
@@ -791,28 +982,18 @@ extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int3
   if (int r = static_scratch_address(c, &base)) return r;
   // the array keeps whatever the previous call (of any context) left: the counters must start at zero
   CU_OK(c, cudaMemsetAsync(base, 0, counters_bytes, c->stream));
-  CU_OK(c, cudaMemcpyAsync(c->fwd_tok, tokens, (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
-  PassDesc pd{};
-  pd.kind = PASS_TOKENS;
-  pd.seq = 0;
-  pd.start = start;
-  pd.count = rows;
-  pd.src = c->fwd_tok;
-  // same pass as sdfp_forward_logits, with the attention scratch pointers swapped for its duration
+  // same passes as sdfp_forward_logits, with the attention scratch pointers swapped for their duration
   float* const own_o = c->part_o;
   float* const own_ml = c->part_ml;
   int* const own_counters = c->attn_counters;
   c->attn_counters = reinterpret_cast<int*>(base);
   c->part_ml = reinterpret_cast<float*>(base + counters_bytes);
   c->part_o = reinterpret_cast<float*>(base + counters_bytes + ml_bytes);
-  const int r = enqueue_pass(c, pd, draft != 0, prow, rps, n_chunks, DECIDE_LOGITS);
+  const int r = forward_logits_passes(c, draft != 0, tokens, rows, start, host_logits);
   c->part_o = own_o;
   c->part_ml = own_ml;
   c->attn_counters = own_counters;
-  if (r) return r;
-  CU_OK(c, cudaMemcpyAsync(host_logits, c->logits, (size_t)rows * g.vocab * 4, cudaMemcpyDeviceToHost, c->stream));
-  CU_OK(c, cudaStreamSynchronize(c->stream));
-  return 0;
+  return r;
 }
 
 extern "C" int sdfp_get_timing(const sdfp_ctx* c, sdfp_timing* out) {

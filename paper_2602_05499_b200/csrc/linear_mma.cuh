@@ -5,8 +5,9 @@
 // kernel is organised around the weight stream, not around the MMA:
 //   * W is re-packed once into 16x16 tiles in the register order of the A operand of
 //     mma.sync.m16n8k16 (out-features on the 16-row side), 512 contiguous bytes per tile,
-//     tiles ordered [row tile][k tile].  A warp loads a tile with ONE 128-bit load per lane,
-//     fully coalesced, straight into MMA registers: no shared-memory staging, no ldmatrix.
+//     tiles ordered [row tile / 8][k tile][row tile % 8] (the unit layout of pass_kernel.cuh,
+//     which both kernels share).  A warp loads a tile with ONE 128-bit load per lane, fully
+//     coalesced, straight into MMA registers: no shared-memory staging, no ldmatrix.
 //   * A CTA owns R row tiles (16·R out-features) over the whole K; its 8 warps split K into 8
 //     contiguous ranges, so every warp reads R sequential streams.  Loads are issued two
 //     batches ahead (register double buffer), the first batch BEFORE griddepcontrol.wait so
@@ -78,7 +79,7 @@ linear_mma_kernel(const uint4* __restrict__ W, const float* __restrict__ X, int 
 #pragma unroll
       for (int r = 0; r < R; ++r) {
         const int kt = ktb + u, rt = rt0 + r;
-        dst[u][r] = (kt < kt1 && rt < NT) ? __ldcs(W + ((size_t)rt * KT + kt) * 32 + lane) : zero4;
+        dst[u][r] = (kt < kt1 && rt < NT) ? __ldcs(W + (((size_t)(rt >> 3) * KT + kt) * 8 + (rt & 7)) * 32 + lane) : zero4;
       }
   };
   auto load_x = [&](XFrag(&dst)[U][CG], int ktb) {
@@ -236,31 +237,6 @@ inline cudaError_t launch_linear_mma(const Launcher& L, int num_sms, const void*
     return launch_mma_t<1, 4, 2>(L, W, X, ldx, M, K, NT, gain, eps, ep);
   }
   return launch_mma_t<1, 8, 1>(L, W, X, ldx, M, K, NT, gain, eps, ep);
-}
-
-// ---- packing into A-fragment tile order --------------------------------------------------
-// element e of the packed buffer: tile t = e / 256 = rt*KT + kt; lane = (e % 256) / 8; j = e % 8:
-//   j = 0,1: (row g,     k 2q + j)        j = 2,3: (row g + 8, k 2q + j - 2)
-//   j = 4,5: (row g,     k 2q + 8 + j-4)  j = 6,7: (row g + 8, k 2q + 8 + j - 6)
-// Row g of tile rt is the first feature of pair 8*rt + g, row g + 8 its second.
-__global__ void pack_mma_kernel(__nv_bfloat16* __restrict__ dst, PackSrc ps, int n_pairs, int K) {
-  const size_t total = (size_t)n_pairs * 2 * K;
-  const int KT = K >> 4;
-  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
-    const size_t t = e >> 8;
-    const int within = (int)(e & 255);
-    const int lane = within >> 3, j = within & 7;
-    const int g = lane >> 2, q = lane & 3;
-    const int rt = (int)(t / KT), kt = (int)(t % KT);
-    const int second = (j >> 1) & 1;
-    const int k = kt * 16 + 2 * q + (j & 1) + ((j >> 2) ? 8 : 0);
-    dst[e] = pack_src_row<__nv_bfloat16>(ps, 8 * rt + g, second, K)[k];
-  }
-}
-
-inline int pack_mma(cudaStream_t stream, __nv_bfloat16* dst, const PackSrc& ps, int n_pairs, int K) {
-  pack_mma_kernel<<<1184, 256, 0, stream>>>(dst, ps, n_pairs, K);
-  return cudaGetLastError() == cudaSuccess ? 0 : -1;
 }
 
 }  // namespace sdfp

@@ -1,0 +1,714 @@
+// Persistent forward-pass kernel for bf16 models (sm_100a): every stage of one pass
+//   per layer [RMSNorm + QKV + RoPE + KV append] [split-KV attention] [O-proj + residual]
+//             [RMSNorm + gate/up + SwiGLU] [down-proj + residual],  then [final RMSNorm + lm-head]
+// runs inside ONE cooperative launch of one CTA per SM.
+//
+// Why one kernel: a decode pass is bound by the bytes of the weights (each is used for at most
+// 16 rows), and a 7B layer is four weight sweeps of 5..28 us each.  As separate launches every
+// sweep pays a ramp-up and a tail; here the weight stream never stops:
+//   * One producer warp per CTA walks the whole stage list and copies this CTA's share of every
+//     weight matrix into a ring of 16 KB shared-memory slots with bulk asynchronous copies
+//     (cp.async.bulk + mbarrier transaction counts).  Weights do not depend on activations, so the
+//     producer runs ahead of the consumers across stage boundaries, through the grid barriers,
+//     as far as the ring allows (160 KB per SM, ~24 MB over the GPU).
+//   * Eight consumer warps take the slots in order, feed the tiles to mma.sync.m16n8k16 (weights
+//     are the A operand, tokens the 8-wide B operand) and run the fused epilogues.
+//   * Stages are separated by a grid barrier (arrival counter in global memory, bounded spin).
+//
+// Weight layout ("unit" layout, written by pack_units_kernel): a matrix with NT 16-row tiles and
+// KT 16-column tiles is stored as units of 8 row tiles at one k-tile, 4096 contiguous bytes,
+// unit index = group * KT + kt with group = row tile / 8; inside a unit tile r at r*512 bytes in
+// the register order of the MMA A fragment.  The units of a matrix are split evenly over the
+// CTAs as contiguous ranges, so every CTA streams one contiguous byte range per stage and the
+// shares differ by at most one unit (4 KB).  A range cuts groups at arbitrary k: a group that
+// spans several CTAs is finished by the CTA that holds its beginning (which reaches it last),
+// after the others have posted their partial sums to global scratch; partials are added in CTA
+// order, so the result does not depend on timing.
+//
+// Inside a CTA the 8 consumer warps are 4 k-classes x 2 tile halves: the unit with index
+// (range start + c + 4i) belongs to class c, and warp (c, t) multiplies its tiles 4t..4t+3.  The
+// four class partials are added in class order through shared memory.  All of this is fixed by
+// the matrix shape and the grid size alone, never by the number of rows, so a row's result is
+// bit-identical whether it is computed alone (autoregressive step) or among k+1 rows (verify).
+#pragma once
+
+#include "attention.cuh"
+#include "common.cuh"
+#include "linear_mma.cuh"
+
+namespace sdfp {
+
+constexpr int kPassConsumerWarps = 8;
+constexpr int kPassConsumerThreads = kPassConsumerWarps * 32;
+constexpr int kPassThreads = kPassConsumerThreads + 32;  // + the producer warp
+constexpr int kUnitTiles = 8;                            // row tiles per unit
+constexpr int kUnitBytes = kUnitTiles * 512;
+constexpr int kChunkUnits = 4;  // units per ring slot = number of k-classes
+constexpr int kSlotBytes = kChunkUnits * kUnitBytes;
+constexpr int kPassMaxRows = 16;  // rows one launch may carry (two column groups of 8)
+constexpr int kPassAttnR = 16;    // rows of one sequence per attention item
+
+enum StageKind { ST_LINEAR = 0, ST_ATTN = 1 };
+
+struct StageDesc {
+  int kind;
+  int K, KT, NT, n_groups;  // linear: in-features, k-tiles, row tiles, groups of 8 row tiles
+  int ldx;
+  const uint4* W;     // unit layout
+  const float* X;     // linear: activations [rows, K]; attention: q [rows, d_model]
+  const float* gain;  // linear: RMSNorm gain or null
+  EpiParams ep;       // linear epilogue; attention: out, kcache, vcache, n_heads, max_seq
+};
+
+// what a wait that gave up leaves in PassSync::error
+enum PassError { PASS_OK = 0, PASS_ERR_GRID_BARRIER = 1, PASS_ERR_SLOT_FULL = 2, PASS_ERR_SLOT_EMPTY = 3, PASS_ERR_SPLIT_FLAG = 4 };
+
+struct PassSync {       // one per context, in global memory, zero-initialised
+  unsigned bar_count;   // grid-barrier arrivals, ever increasing (wraps)
+  unsigned bar_base;    // value of bar_count when the running launch started
+  unsigned epoch_base;  // serial number of the last stage of the previous launch
+  int error;            // first PassError seen, sticky
+};
+
+struct PassParams {
+  const StageDesc* prog;
+  int n_stages;
+  int M;             // rows in this pass (<= kPassMaxRows); rows beyond carry nothing
+  int rows_per_seq;  // attention: rows m0..m0+R-1 of a group belong to one sequence
+  int n_chunks;      // attention: 64-key chunks that bound the context
+  const int* row_pos;
+  const int* row_seq;
+  float eps;
+  float attn_scale;
+  // scratch
+  float* part_o;          // attention partials [rows][head][chunk][head_dim]
+  float* part_ml;         // [rows][head][chunk][2]
+  int* attn_counters;     // [groups][head], zero between launches
+  float* split_partials;  // [grid][kUnitTiles * CG * 64 * 2]
+  unsigned* split_flags;  // [grid]
+  PassSync* sync;
+};
+
+// ---- PTX helpers ---------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
+  asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(smem_u32(bar)), "r"(bytes)
+               : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
+  unsigned ok;
+  asm volatile(
+      "{\n .reg .pred p;\n mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n selp.u32 %0, 1, 0, p;\n}"
+      : "=r"(ok)
+      : "r"(smem_u32(bar)), "r"(parity)
+      : "memory");
+  return ok != 0;
+}
+// Bulk asynchronous copy global -> shared, completion counted in bytes on an mbarrier.
+// Both addresses and the size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+               : "memory");
+}
+__device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
+  unsigned v;
+  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
+  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
+  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+}
+__device__ __forceinline__ unsigned long long global_ns() {
+  unsigned long long t;
+  asm volatile("mov.u64 %0, %globaltimer;" : "=l"(t));
+  return t;
+}
+__device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kPassConsumerThreads) : "memory"); }
+__device__ __forceinline__ void half_sync(int half) { asm volatile("bar.sync %0, 128;" ::"r"(2 + half) : "memory"); }
+
+// Every wait in this kernel gives up after this long, records why, and the kernel winds down.
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct PassShared {
+  uint64_t full[16];
+  uint64_t empty[16];
+  StageDesc st;  // the running stage, copied once per stage by the consumer threads
+  float inv_rms[kPassMaxRows];
+  int abort;     // set by whichever thread gives up a wait
+  int decision;  // abort as sampled by thread 0 between two consumer barriers: uniform for all
+  int attn_pos[2][kPassAttnR];
+  int attn_last[2];
+  int n_parts;
+  int parts[160];  // CTAs that post a partial for the group this CTA finishes
+};
+
+// All consumer threads learn the same answer to "has anything failed": thread 0 samples the
+// flag between two barriers, so warps never disagree about leaving a loop that contains barriers.
+__device__ __forceinline__ bool consumers_agree_ok(PassShared* sh) {
+  consumer_sync();
+  if (threadIdx.x == 0) sh->decision = sh->abort;
+  consumer_sync();
+  return sh->decision == 0;
+}
+
+// Spin until pred() holds; false (and the error recorded) if the limit passes or another CTA
+// has already failed.
+template <typename Pred>
+__device__ __forceinline__ bool bounded_wait(Pred pred, PassSync* sync, volatile int* s_abort, int code) {
+  if (pred()) return true;
+  const unsigned long long t0 = global_ns();
+  unsigned spins = 0;
+  for (;;) {
+    if (pred()) return true;
+    if (((++spins) & 255u) == 0) {
+      if (*s_abort) return false;
+      if (*reinterpret_cast<volatile int*>(&sync->error) != 0) {
+        *s_abort = 1;
+        return false;
+      }
+      if (global_ns() - t0 > kWaitLimitNs) {
+        atomicCAS(&sync->error, 0, code);
+        *s_abort = 1;
+        return false;
+      }
+    }
+  }
+}
+
+// ---- grid barrier (consumer threads of every CTA) ------------------------------------------------
+// Everything the consumer threads of this CTA wrote before is visible to every CTA after.
+__device__ __forceinline__ bool grid_barrier(PassSync* sync, unsigned target, PassShared* sh) {
+  consumer_sync();
+  if (threadIdx.x == 0) {
+    __threadfence();
+    red_release_add(&sync->bar_count, 1u);
+    bounded_wait([&] { return (int)(ld_acquire(&sync->bar_count) - target) >= 0; }, sync, &sh->abort, PASS_ERR_GRID_BARRIER);
+    sh->decision = sh->abort;
+  }
+  consumer_sync();
+  return sh->decision == 0;
+}
+
+__device__ __forceinline__ void unit_range(long long n_units, int cta, int n_cta, long long& ub, long long& ue) {
+  ub = n_units * cta / n_cta;
+  ue = n_units * (cta + 1) / n_cta;
+}
+
+// ---- one linear stage, consumer side -------------------------------------------------------------
+template <int CG>
+struct XRegs {
+  float2 lo8[CG], hi8[CG];
+};
+
+template <int CG>
+__device__ __forceinline__ void load_xregs(XRegs<CG>& x, const float* X, int ldx, int M, int kt, int g, int q, bool valid) {
+#pragma unroll
+  for (int cg = 0; cg < CG; ++cg) {
+    const int m = cg * 8 + g;
+    x.lo8[cg] = make_float2(0.f, 0.f);
+    x.hi8[cg] = make_float2(0.f, 0.f);
+    if (valid && m < M) {
+      const float* xp = X + (size_t)m * ldx + kt * 16 + 2 * q;
+      x.lo8[cg] = ld_act2(xp);
+      x.hi8[cg] = ld_act2(xp + 8);
+    }
+  }
+}
+
+template <int CG>
+__device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigned char* ring, int n_slots, float4* red,
+                             unsigned& chunk_base, unsigned epoch) {
+  const StageDesc& st = sh->st;
+  const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
+  const int g = lane >> 2, q = lane & 3;
+  const int cls = warp & 3, th = warp >> 2;
+  const int KT = st.KT, M = pp.M, ldx = st.ldx;
+  const float* const X = st.X;
+  const float* const gain = st.gain;
+  const int cta = blockIdx.x, n_cta = gridDim.x;
+  const long long n_units = (long long)st.n_groups * KT;
+  long long ub64, ue64;
+  unit_range(n_units, cta, n_cta, ub64, ue64);
+  const int nun = (int)(ue64 - ub64);  // units of this CTA; below, units are numbered from ub64
+  const int n_chunks = (nun + kChunkUnits - 1) / kChunkUnits;
+  const int my_n = nun > cls ? (nun - cls + kChunkUnits - 1) / kChunkUnits : 0;
+  const int grp0 = (int)(ub64 / KT);
+  const int kt_first = (int)(ub64 - (long long)grp0 * KT);  // k-tile of unit 0
+
+  // 1/rms of every row: the same fixed-order sum in every CTA
+  if (gain != nullptr) {
+    float* s_part = reinterpret_cast<float*>(red);  // [warp][row]
+    for (int m = 0; m < M; ++m) {
+      const float* x = X + (size_t)m * ldx;
+      float s = 0.f;
+      for (int k = tid * 4; k < st.K; k += kPassConsumerThreads * 4) {
+        const float4 v = ld_act4(x + k);
+        s = fmaf(v.x, v.x, s);
+        s = fmaf(v.y, v.y, s);
+        s = fmaf(v.z, v.z, s);
+        s = fmaf(v.w, v.w, s);
+      }
+      s = warp_sum(s);
+      if (lane == 0) s_part[warp * kPassMaxRows + m] = s;
+    }
+    consumer_sync();
+    if (tid < M) {
+      float s = 0.f;
+#pragma unroll
+      for (int w = 0; w < kPassConsumerWarps; ++w) s += s_part[w * kPassMaxRows + tid];
+      sh->inv_rms[tid] = rsqrtf(s / (float)st.K + pp.eps);
+    }
+  } else if (tid < kPassMaxRows) {
+    sh->inv_rms[tid] = 1.f;
+  }
+  consumer_sync();
+
+  // activation fragments of my next four units; kt_pref = k-tile of the next unit to prefetch
+  XRegs<CG> x0, x1, x2, x3;
+  int kt_pref = (kt_first + cls) % KT;
+  auto prefetch = [&](XRegs<CG>& x, int i) {
+    load_xregs<CG>(x, X, ldx, M, kt_pref, g, q, i < my_n);
+    kt_pref += kChunkUnits;
+    if (kt_pref >= KT) kt_pref -= KT;
+  };
+  prefetch(x0, 0);
+  prefetch(x1, 1);
+  prefetch(x2, 2);
+  prefetch(x3, 3);
+
+  int i = 0;          // my next unit is number cls + 4 i
+  int seg_begin = 0;  // in units from ub64
+  int grp = grp0;
+  int seg_kt0 = kt_first;  // k-tile at seg_begin
+  while (seg_begin < nun) {
+    const int seg_len = min(nun - seg_begin, KT - seg_kt0);
+    const int seg_end = seg_begin + seg_len;
+    float acc[4][CG][4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int cg = 0; cg < CG; ++cg)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[r][cg][e] = 0.f;
+
+    bool warp_ok = true;
+    while (warp_ok && i < my_n && cls + kChunkUnits * i < seg_end) {
+      const int kt = seg_kt0 + (cls + kChunkUnits * i - seg_begin);
+      const unsigned gc = chunk_base + (unsigned)i;
+      const unsigned slot = gc % (unsigned)n_slots, parity = (gc / (unsigned)n_slots) & 1u;
+      // Lanes leave the polling loop at different times.  mma.sync needs the whole warp
+      // converged, so the vote below is both the warp-uniform outcome and the reconvergence point.
+      warp_ok = __all_sync(0xffffffffu, bounded_wait([&] { return mbar_try_wait(&sh->full[slot], parity); }, pp.sync,
+                                                     &sh->abort, PASS_ERR_SLOT_FULL));
+      if (!warp_ok) break;
+      const uint4* tiles = reinterpret_cast<const uint4*>(ring + (size_t)slot * kSlotBytes + cls * kUnitBytes + th * 4 * 512);
+      uint4 a[4];
+#pragma unroll
+      for (int r = 0; r < 4; ++r) a[r] = tiles[r * 32 + lane];
+      float2 g0 = make_float2(1.f, 1.f), g1 = make_float2(1.f, 1.f);
+      if (gain != nullptr) {
+        const float* gp = gain + kt * 16 + 2 * q;
+        g0 = *reinterpret_cast<const float2*>(gp);
+        g1 = *reinterpret_cast<const float2*>(gp + 8);
+      }
+#pragma unroll
+      for (int cg = 0; cg < CG; ++cg) {
+        uint32_t bh0, bl0, bh1, bl1;
+        split_pack(x0.lo8[cg].x * g0.x, x0.lo8[cg].y * g0.y, bh0, bl0);
+        split_pack(x0.hi8[cg].x * g1.x, x0.hi8[cg].y * g1.y, bh1, bl1);
+#pragma unroll
+        for (int r = 0; r < 4; ++r) {
+          mma_bf16_16816(acc[r][cg], a[r], bh0, bh1);
+          mma_bf16_16816(acc[r][cg], a[r], bl0, bl1);
+        }
+      }
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->empty[slot]);
+      x0 = x1;
+      x1 = x2;
+      x2 = x3;
+      prefetch(x3, i + 4);
+      ++i;
+    }
+
+    // ---- end of the segment: add the four class partials, then finish the group or post ----
+#pragma unroll
+    for (int r = 0; r < 4; ++r)
+#pragma unroll
+      for (int cg = 0; cg < CG; ++cg)
+        red[((cls * kUnitTiles + th * 4 + r) * CG + cg) * 32 + lane] =
+            make_float4(acc[r][cg][0], acc[r][cg][1], acc[r][cg][2], acc[r][cg][3]);
+    const bool starts_group = (seg_kt0 == 0);
+    const bool whole = starts_group && (seg_len == KT);
+    const bool owner = starts_group && !whole;
+    if (owner && tid == 0) {
+      // the rest of the group sits at the beginning of the ranges of the CTAs that follow
+      const long long grp_end = (long long)(grp + 1) * KT;
+      int n = 0;
+      bool w_ok = true;
+      for (int c2 = cta + 1; c2 < n_cta && w_ok; ++c2) {
+        long long b2, e2;
+        unit_range(n_units, c2, n_cta, b2, e2);
+        if (b2 >= grp_end) break;
+        if (e2 == b2) continue;  // an empty range posts nothing
+        sh->parts[n++] = c2;
+        w_ok = bounded_wait([&] { return ld_acquire(pp.split_flags + c2) == epoch; }, pp.sync, &sh->abort, PASS_ERR_SPLIT_FLAG);
+      }
+      sh->n_parts = n;
+    }
+    if (!consumers_agree_ok(sh)) return;
+
+    {
+      float2* my_post = reinterpret_cast<float2*>(pp.split_partials) + (size_t)cta * (kUnitTiles * CG * 64);
+      const int n_parts = owner ? sh->n_parts : 0;
+      for (int it = tid; it < kUnitTiles * CG * 64; it += kPassConsumerThreads) {
+        const int ch = it & 1;
+        const int ln = (it >> 1) & 31;
+        const int rc = it >> 6;
+        const int cg = rc % CG, tile = rc / CG;
+        float v0 = 0.f, v1 = 0.f;
+#pragma unroll
+        for (int c4 = 0; c4 < 4; ++c4) {
+          const float* p = reinterpret_cast<const float*>(red + ((c4 * kUnitTiles + tile) * CG + cg) * 32 + ln);
+          v0 += p[ch];
+          v1 += p[ch + 2];
+        }
+        if (!starts_group) {
+          my_post[it] = make_float2(v0, v1);
+          continue;
+        }
+        for (int j = 0; j < n_parts; ++j) {
+          const float2 o =
+              __ldcg(reinterpret_cast<const float2*>(pp.split_partials) + (size_t)sh->parts[j] * (kUnitTiles * CG * 64) + it);
+          v0 += o.x;
+          v1 += o.y;
+        }
+        const int m = cg * 8 + 2 * (ln & 3) + ch;
+        const int rt = grp * kUnitTiles + tile;
+        if (m < M && rt < st.NT) {
+          const float inv = sh->inv_rms[m];
+          apply_epilogue<__nv_bfloat16>(st.ep, 8 * rt + (ln >> 2), m, v0 * inv, v1 * inv);
+        }
+      }
+    }
+    if (!starts_group) __threadfence();  // every thread publishes its own part of the partial sum
+    consumer_sync();                     // red and parts may be rewritten; the partial is complete
+    if (!starts_group && tid == 0) {
+      __threadfence();
+      st_release(pp.split_flags + cta, epoch);
+    }
+    seg_begin = seg_end;
+    seg_kt0 = 0;
+    ++grp;
+  }
+  // A class without a unit in the last, partial slot still has to hand that slot back, and only
+  // once the slot has been filled: an earlier arrival would be counted for the slot's previous
+  // use and let the producer overwrite tiles another warp is still reading.
+  if (my_n < n_chunks) {
+    const unsigned gc = chunk_base + (unsigned)(n_chunks - 1);
+    const unsigned slot = gc % (unsigned)n_slots, parity = (gc / (unsigned)n_slots) & 1u;
+    if (bounded_wait([&] { return mbar_try_wait(&sh->full[slot], parity); }, pp.sync, &sh->abort, PASS_ERR_SLOT_FULL)) {
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&sh->empty[slot]);
+    }
+  }
+  chunk_base += (unsigned)n_chunks;
+}
+
+// ---- attention stage: one item = (64-key chunk, head, row group), handled by half a CTA -------------
+template <int HD>
+__device__ void attention_item(const StageDesc& st, const PassParams& pp, PassShared* sh, unsigned char* smem, int half,
+                               int htid, int c, int head, int b) {
+  using KT = __nv_bfloat16;
+  constexpr int C = kAttnChunk;
+  KT* sV = reinterpret_cast<KT*>(smem);               // [C][HD]
+  float* sQ = reinterpret_cast<float*>(sV + C * HD);  // [R][HD]
+  float* sS = sQ + kPassAttnR * HD;                   // [R][C]
+  int* s_pos = sh->attn_pos[half];
+  const int R = pp.rows_per_seq;
+  const int row0 = b * R;
+  const int key0 = c * C;
+  const int n_heads = st.ep.n_heads;
+  const size_t d_model = (size_t)n_heads * HD;
+
+  if (htid < R) s_pos[htid] = (row0 + htid < pp.M) ? ld_act(pp.row_pos + row0 + htid) : -1;
+  half_sync(half);
+  int max_pos = -1;
+  for (int i = 0; i < R; ++i) max_pos = max(max_pos, s_pos[i]);
+
+  if (max_pos >= key0) {
+    const int seq = ld_act(pp.row_seq + row0);
+    const int nk_all = min(C, max_pos + 1 - key0);
+    const size_t base = (((size_t)seq * n_heads + head) * st.ep.max_seq + key0) * HD;
+    const KT* gK = reinterpret_cast<const KT*>(st.ep.kcache) + base;
+    const KT* gV = reinterpret_cast<const KT*>(st.ep.vcache) + base;
+    // this thread's half of one key row goes straight to registers
+    constexpr int KV4 = HD / 16;  // uint4 per half row
+    const int key = htid >> 1, hf = htid & 1;
+    uint4 kreg[KV4];
+#pragma unroll
+    for (int j = 0; j < KV4; ++j) kreg[j] = make_uint4(0u, 0u, 0u, 0u);
+    if (key < nk_all) {
+      const uint4* kp = reinterpret_cast<const uint4*>(gK + (size_t)key * HD + hf * (HD / 2));
+#pragma unroll
+      for (int j = 0; j < KV4; ++j) kreg[j] = __ldcg(kp + j);
+    }
+    constexpr int VPR = HD / 8;
+    for (int v = htid; v < nk_all * VPR; v += 128)
+      reinterpret_cast<uint4*>(sV)[v] = __ldcg(reinterpret_cast<const uint4*>(gV) + v);
+    for (int e = htid; e < R * HD; e += 128) {
+      const int i = e / HD, d = e - i * HD;
+      sQ[e] = (s_pos[i] >= 0) ? ld_act(st.X + (size_t)(row0 + i) * d_model + head * HD + d) : 0.f;
+    }
+    half_sync(half);
+
+    {
+      float acc[kPassAttnR];
+#pragma unroll
+      for (int i = 0; i < kPassAttnR; ++i) acc[i] = 0.f;
+      const float* qh = sQ + hf * (HD / 2);
+#pragma unroll
+      for (int j = 0; j < KV4; ++j) {
+        const uint32_t w[4] = {kreg[j].x, kreg[j].y, kreg[j].z, kreg[j].w};
+#pragma unroll
+        for (int e = 0; e < 4; ++e) {
+          const float k0 = __uint_as_float(w[e] << 16), k1 = __uint_as_float(w[e] & 0xffff0000u);
+          const int d = j * 8 + e * 2;
+#pragma unroll
+          for (int i = 0; i < kPassAttnR; ++i) {
+            if (i < R) {
+              const float2 qv = *reinterpret_cast<const float2*>(qh + i * HD + d);
+              acc[i] = fmaf(k0, qv.x, acc[i]);
+              acc[i] = fmaf(k1, qv.y, acc[i]);
+            }
+          }
+        }
+      }
+#pragma unroll
+      for (int i = 0; i < kPassAttnR; ++i) {
+        if (i < R) {
+          const float other = __shfl_xor_sync(0xffffffffu, acc[i], 1);
+          if (hf == 0) sS[i * C + key] = (acc[i] + other) * pp.attn_scale;
+        }
+      }
+    }
+    half_sync(half);
+
+    {
+      const int w4 = htid >> 5, lane = htid & 31;
+      for (int i = w4; i < R; i += 4) {
+        const int nk = min(C, s_pos[i] + 1 - key0);
+        const float s0 = (lane < nk) ? sS[i * C + lane] : -INFINITY;
+        const float s1 = (lane + 32 < nk) ? sS[i * C + lane + 32] : -INFINITY;
+        const float mx = warp_max(fmaxf(s0, s1));
+        const float p0 = (lane < nk) ? __expf(s0 - mx) : 0.f;
+        const float p1 = (lane + 32 < nk) ? __expf(s1 - mx) : 0.f;
+        sS[i * C + lane] = p0;
+        sS[i * C + lane + 32] = p1;
+        const float l = warp_sum(p0 + p1);
+        if (lane == 0 && nk > 0) {
+          float* ml = pp.part_ml + ((((size_t)(row0 + i)) * n_heads + head) * pp.n_chunks + c) * 2;
+          ml[0] = mx;
+          ml[1] = l;
+        }
+      }
+    }
+    half_sync(half);
+
+    for (int d = htid; d < HD; d += 128) {
+      float o[kPassAttnR];
+#pragma unroll
+      for (int i = 0; i < kPassAttnR; ++i) o[i] = 0.f;
+      for (int k2 = 0; k2 < nk_all; ++k2) {
+        const float v = __bfloat162float(sV[k2 * HD + d]);
+#pragma unroll
+        for (int i = 0; i < kPassAttnR; ++i)
+          if (i < R) o[i] = fmaf(sS[i * C + k2], v, o[i]);
+      }
+#pragma unroll
+      for (int i = 0; i < kPassAttnR; ++i)
+        if (i < R && s_pos[i] >= key0)
+          pp.part_o[((((size_t)(row0 + i)) * n_heads + head) * pp.n_chunks + c) * HD + d] = o[i];
+    }
+  }
+
+  // the half-CTA that arrives last for this (group, head) folds the chunks in chunk order
+  __threadfence();
+  half_sync(half);
+  if (htid == 0) {
+    const int prev = atomicAdd(&pp.attn_counters[b * n_heads + head], 1);
+    sh->attn_last[half] = (prev == pp.n_chunks - 1);
+  }
+  half_sync(half);
+  if (sh->attn_last[half]) {
+    __threadfence();
+    if (htid == 0) pp.attn_counters[b * n_heads + head] = 0;
+    for (int i = 0; i < R; ++i) {
+      if (row0 + i >= pp.M) break;
+      const int pos = s_pos[i];
+      float* dst = st.ep.out + (size_t)(row0 + i) * d_model + head * HD;
+      if (pos < 0) {
+        for (int d = htid; d < HD; d += 128) dst[d] = 0.f;
+        continue;
+      }
+      const int nc = pos / C + 1;
+      const float* ml = pp.part_ml + (((size_t)(row0 + i)) * n_heads + head) * pp.n_chunks * 2;
+      const float* po = pp.part_o + (((size_t)(row0 + i)) * n_heads + head) * pp.n_chunks * HD;
+      float mx = -INFINITY;
+      for (int cc = 0; cc < nc; ++cc) mx = fmaxf(mx, __ldcg(ml + cc * 2));
+      float l = 0.f;
+      for (int cc = 0; cc < nc; ++cc) l = fmaf(__ldcg(ml + cc * 2 + 1), __expf(__ldcg(ml + cc * 2) - mx), l);
+      const float inv_l = 1.0f / l;
+      for (int d = htid; d < HD; d += 128) {
+        float o = 0.f;
+        for (int cc = 0; cc < nc; ++cc) o = fmaf(__ldcg(po + (size_t)cc * HD + d), __expf(__ldcg(ml + cc * 2) - mx), o);
+        dst[d] = o * inv_l;
+      }
+    }
+  }
+  half_sync(half);  // smem and s_pos are reused by the next item
+}
+
+template <int HD>
+__host__ __device__ constexpr size_t pass_attn_smem_half() {
+  return (size_t)kAttnChunk * HD * 2 + (size_t)kPassAttnR * HD * 4 + (size_t)kPassAttnR * kAttnChunk * 4;
+}
+
+template <int CG>
+__host__ __device__ constexpr size_t pass_red_bytes() {
+  return (size_t)4 * kUnitTiles * CG * 32 * sizeof(float4);
+}
+
+template <int CG, int HD>
+__host__ __device__ constexpr size_t pass_work_bytes() {
+  return pass_red_bytes<CG>() > 2 * pass_attn_smem_half<HD>() ? pass_red_bytes<CG>() : 2 * pass_attn_smem_half<HD>();
+}
+
+// Dynamic shared memory: [ring: n_slots * 16 KB][work area: reduction buffer / attention tiles][PassShared]
+template <int CG, int HD>
+__global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, int n_slots) {
+  extern __shared__ __align__(1024) unsigned char smem[];
+  unsigned char* ring = smem;
+  unsigned char* work = smem + (size_t)n_slots * kSlotBytes;
+  PassShared* sh = reinterpret_cast<PassShared*>(work + pass_work_bytes<CG, HD>());
+  const int tid = threadIdx.x;
+
+  if (tid == 0) {
+    for (int s = 0; s < n_slots; ++s) {
+      mbar_init(&sh->full[s], 1);
+      mbar_init(&sh->empty[s], kPassConsumerWarps);
+    }
+    sh->abort = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+  }
+  __syncthreads();
+
+  if (tid >= kPassConsumerThreads) {
+    // ================= producer warp: stream this CTA's share of every weight matrix =================
+    if (tid == kPassConsumerThreads) {
+      unsigned gc = 0;
+      bool ok = true;
+      for (int s = 0; s < pp.n_stages && ok; ++s) {
+        const StageDesc& st = pp.prog[s];
+        if (st.kind != ST_LINEAR) continue;
+        long long ub, ue;
+        unit_range((long long)st.n_groups * st.KT, blockIdx.x, gridDim.x, ub, ue);
+        const unsigned char* src = reinterpret_cast<const unsigned char*>(st.W) + (size_t)ub * kUnitBytes;
+        long long left = ue - ub;
+        while (left > 0) {
+          const unsigned slot = gc % (unsigned)n_slots, parity = ((gc / (unsigned)n_slots) & 1u) ^ 1u;
+          ok = bounded_wait([&] { return mbar_try_wait(&sh->empty[slot], parity); }, pp.sync, &sh->abort, PASS_ERR_SLOT_EMPTY);
+          if (!ok) break;
+          const unsigned n = left < kChunkUnits ? (unsigned)left : (unsigned)kChunkUnits;
+          mbar_arrive_expect_tx(&sh->full[slot], n * kUnitBytes);
+          bulk_load(ring + (size_t)slot * kSlotBytes, src, n * kUnitBytes, &sh->full[slot]);
+          src += (size_t)n * kUnitBytes;
+          left -= n;
+          ++gc;
+        }
+      }
+      // nothing may still be landing in shared memory when the CTA exits: wait (bounded) for the
+      // copies of the last n_slots slots that were issued
+      const unsigned first = gc > (unsigned)n_slots ? gc - (unsigned)n_slots : 0u;
+      for (unsigned j = first; j < gc; ++j) {
+        const unsigned slot = j % (unsigned)n_slots, parity = (j / (unsigned)n_slots) & 1u;
+        const unsigned long long t0 = global_ns();
+        while (!mbar_try_wait(&sh->full[slot], parity))
+          if (global_ns() - t0 > kWaitLimitNs) break;
+      }
+    }
+    return;
+  }
+
+  // ================= consumer warps =================
+  const unsigned bar_base = *reinterpret_cast<volatile unsigned*>(&pp.sync->bar_base);
+  const unsigned epoch_base = *reinterpret_cast<volatile unsigned*>(&pp.sync->epoch_base);
+  unsigned chunk_base = 0;
+  float4* red = reinterpret_cast<float4*>(work);
+  bool ok = true;
+  for (int s = 0; s < pp.n_stages && ok; ++s) {
+    {
+      const int* src = reinterpret_cast<const int*>(pp.prog + s);
+      int* dst = reinterpret_cast<int*>(&sh->st);
+      for (int w = tid; w < (int)(sizeof(StageDesc) / sizeof(int)); w += kPassConsumerThreads) dst[w] = src[w];
+      consumer_sync();
+    }
+    if (sh->st.kind == ST_LINEAR) {
+      linear_stage<CG>(pp, sh, ring, n_slots, red, chunk_base, epoch_base + (unsigned)s + 1u);
+    } else {
+      const int half = tid >> 7, htid = tid & 127;
+      const int n_heads = sh->st.ep.n_heads;
+      const int n_groups = (pp.M + pp.rows_per_seq - 1) / pp.rows_per_seq;
+      const int items = pp.n_chunks * n_heads * n_groups;
+      unsigned char* my = work + (size_t)half * pass_attn_smem_half<HD>();
+      for (int it = blockIdx.x * 2 + half; it < items; it += gridDim.x * 2) {
+        const int c = it % pp.n_chunks;
+        const int hb = it / pp.n_chunks;
+        attention_item<HD>(sh->st, pp, sh, my, half, htid, c, hb % n_heads, hb / n_heads);
+      }
+    }
+    ok = consumers_agree_ok(sh);
+    if (ok && s + 1 < pp.n_stages) ok = grid_barrier(pp.sync, bar_base + (unsigned)(s + 1) * gridDim.x, sh);
+  }
+  // the next launch starts from where this one ended (written after the last barrier, read by
+  // every CTA before its first one)
+  if (blockIdx.x == 0 && tid == 0 && ok) {
+    pp.sync->bar_base = bar_base + (unsigned)(pp.n_stages - 1) * gridDim.x;
+    pp.sync->epoch_base = epoch_base + (unsigned)pp.n_stages;
+  }
+}
+
+// ---- packing into the unit layout -----------------------------------------------------------------
+// element e: unit = e / 2048 = group * KT + kt; tile r = (e % 2048) / 256; inside the tile the
+// register order of the MMA A fragment: lane = (e % 256) / 8, j = e % 8,
+//   j = 0,1: (row g,     k 2q + j)        j = 2,3: (row g + 8, k 2q + j - 2)
+//   j = 4,5: (row g,     k 2q + 8 + j-4)  j = 6,7: (row g + 8, k 2q + 8 + j - 6)
+// Row g of tile rt is the first feature of pair 8*rt + g, row g + 8 its second.  Row tiles
+// beyond NT (a ragged last group) are zero.
+__global__ void pack_units_kernel(__nv_bfloat16* __restrict__ dst, PackSrc ps, int n_pairs, int K, int n_groups) {
+  const int KT = K >> 4, NT = n_pairs >> 3;
+  const size_t total = (size_t)n_groups * KT * (kUnitBytes / 2);
+  for (size_t e = (size_t)blockIdx.x * blockDim.x + threadIdx.x; e < total; e += (size_t)gridDim.x * blockDim.x) {
+    const size_t unit = e >> 11;
+    const int within = (int)(e & 2047);
+    const int r = within >> 8, lane = (within & 255) >> 3, j = within & 7;
+    const int grp = (int)(unit / KT), kt = (int)(unit % KT);
+    const int rt = grp * kUnitTiles + r;
+    const int g = lane >> 2, q = lane & 3;
+    const int second = (j >> 1) & 1;
+    const int k = kt * 16 + 2 * q + (j & 1) + ((j >> 2) ? 8 : 0);
+    dst[e] = rt < NT ? pack_src_row<__nv_bfloat16>(ps, 8 * rt + g, second, K)[k] : __float2bfloat16_rn(0.f);
+  }
+}
+
+}  // namespace sdfp

@@ -275,6 +275,30 @@ def test_greedy_7b_shape(l7b4, k):
             assert out.stats[:, 0, 1].tolist() == [r.accepted for r in ref.rounds]
 
 
+@pytest.mark.parametrize("shape,draw", [(si.TINY_BF16, "cpu"), (si.LLAMA7B_4L, "cuda:0")])
+def test_per_operation_kernels_agree_with_pass_kernel(shape, draw):
+    """bf16 models run whole passes in one persistent kernel; with SDFP_FLAG_NO_PASS_KERNEL the
+    same model runs one kernel per operation.  Both must match the oracle, agree closely with
+    each other, and the per-operation path must keep speculative == autoregressive."""
+    toks = si.make_prompts(shape.vocab, 1, 40, seed=14)[0].tolist()
+    prompt = si.make_prompts(shape.vocab, 1, 20, seed=15)
+    e1, m, _ = make_pair(shape, (1, 2), max_seq=128, draw_device=draw)
+    a = e1.sdfp_forward_logits(toks, 0)
+    g1 = e1.sdfp_generate(prompt, 4, 24)
+    e1.close()
+    e2, _, _ = make_pair(shape, (1, 2), max_seq=128, flags=pkg.FLAG_NO_PASS_KERNEL, draw_device=draw)
+    b = e2.sdfp_forward_logits(toks, 0)
+    g2 = e2.sdfp_generate(prompt, 4, 24)
+    ar2 = e2.sdfp_generate(prompt, 0, 24)
+    e2.close()
+    ref = orc.CachedLM(m, max_seq=128).feed(toks, 0).numpy()
+    assert rel_l2(a, ref) < 1e-2 and rel_l2(b, ref) < 1e-2
+    assert rel_l2(a, b) < 2e-3
+    assert g2.tokens == ar2.tokens
+    check_stream_against_oracle(m, prompt[0].tolist(), g1.tokens[0])
+    check_stream_against_oracle(m, prompt[0].tolist(), g2.tokens[0])
+
+
 def test_fma_and_tensor_paths_agree_closely():
     """The CUDA-core comparison path and the tensor-core path compute the same model."""
     shape = si.LLAMA7B_4L
