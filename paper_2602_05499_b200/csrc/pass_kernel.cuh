@@ -332,6 +332,11 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
           mma_bf16_16816(acc[r][cg], a[r], bl0, bl1);
         }
       }
+      // The tiles were read through the generic proxy; the slot is about to be handed back to
+      // the producer, whose next bulk copy writes it through the async proxy.  Without this
+      // fence the arrival could take effect while the reads were still pending, and a refill
+      // then replaced 64-byte pieces of a tile under them (seen as rare wrong rows at full speed).
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->empty[slot]);
       x0 = x1;
