@@ -178,11 +178,12 @@ int sdfp_forward_logits(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int
  *
  * Arguments, results and errors are those of sdfp_forward_logits, and the logits are the same
  * bit for bit.  In addition:
- *   - SDFP_EINVAL when R x n_heads x ceil((start + rows) / 64) x (head_dim + 2) x 4 bytes,
- *     plus the counters, exceed SDFP_STATIC_SCRATCH_BYTES, where R is the number of rows of
- *     the widest pass the call runs (rows, but at most 16 for bf16 models, which are served
- *     in passes of 16 rows; rounded up to a multiple of 16 beyond 16).  The message states
- *     both sizes.
+ *   - SDFP_EINVAL when R x n_heads x P x (head_dim + 2) x 4 bytes, plus the counters, exceed
+ *     SDFP_STATIC_SCRATCH_BYTES.  R is the number of rows of the widest pass the call runs and
+ *     P the number of partials per (row, head): for bf16 models on the whole-pass kernel
+ *     R <= 16 and P = 8, which always fits; with SDFP_FLAG_NO_PASS_KERNEL, with
+ *     SDFP_FLAG_FMA_GEMM and for fp32 models R = rows (rounded up to a multiple of 16 beyond
+ *     16) and P = ceil((start + rows) / 64).  The message states both sizes.
  *   - The first call on a device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and keeps it.  Make that first call
  *     before starting any stream capture.

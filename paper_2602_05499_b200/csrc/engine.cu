@@ -97,6 +97,7 @@ struct sdfp_ctx {
   PassSync* psync = nullptr;
   float* split_partials = nullptr;
   unsigned* split_flags = nullptr;
+  float* ssq_part = nullptr;
   int pass_slots = 0;
   size_t pass_smem = 0;
   int pass_grid = 0;
@@ -242,6 +243,9 @@ StageDesc linear_desc(const void* w, const float* x, int K, int n_pairs, const f
   s.NT = n_pairs / 8;
   s.n_groups = (s.NT + kUnitTiles - 1) / kUnitTiles;
   s.ldx = K;
+  s.x_mode = X_PLAIN;
+  s.rms_mode = gain ? RMS_FROM_PARTS : RMS_NONE;
+  s.write_ssq = ep.mode == EPI_RESID ? 1 : 0;
   s.W = reinterpret_cast<const uint4*>(w);
   s.X = x;
   s.gain = gain;
@@ -255,6 +259,7 @@ StageDesc linear_desc(const void* w, const float* x, int K, int n_pairs, const f
 int build_program(sdfp_ctx* c, bool draft, StageDesc** dev, int* n_out) {
   const sdfp_config& g = c->cfg;
   const int d = g.d_model, f = g.d_ffn;
+  const int resid_groups = (d / 16 + kUnitTiles - 1) / kUnitTiles;  // groups of the stages that write the residual stream
   const KvCache& kv = draft ? c->cache_d : c->cache_t;
   std::vector<StageDesc> prog;
   for (int l = 0; l < g.n_layers; ++l) {
@@ -264,18 +269,23 @@ int build_program(sdfp_ctx* c, bool draft, StageDesc** dev, int* n_out) {
     qkv.kcache = kv.k[l];
     qkv.vcache = kv.v[l];
     prog.push_back(linear_desc(lw.qkv, c->h, d, 3 * d / 2, lw.attn_gain, qkv));
+    // the embedding rows come from another kernel: the first norm of a pass sums its rows itself
+    if (prog.size() == 1) prog.back().rms_mode = RMS_DIRECT;
     StageDesc at{};
     at.kind = ST_ATTN;
     at.X = c->q;
-    at.ep = base_epi(c, EPI_RESID, c->att, d);
+    at.ep = base_epi(c, EPI_RESID, nullptr, d);
     at.ep.kcache = kv.k[l];
     at.ep.vcache = kv.v[l];
     prog.push_back(at);
-    prog.push_back(linear_desc(lw.wo, c->att, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+    // the O-projection reads the attention output as kAttnSplits partials per (row, head)
+    prog.push_back(linear_desc(lw.wo, nullptr, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+    prog.back().x_mode = X_ATTN_FOLD;
     prog.push_back(linear_desc(lw.gu, c->h, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
     prog.push_back(linear_desc(lw.down, c->u, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
   }
   prog.push_back(linear_desc(c->lm_head, c->h, d, g.vocab / 2, c->final_gain, base_epi(c, EPI_LOGITS, c->logits, g.vocab)));
+  for (StageDesc& sd : prog) sd.ssq_groups = resid_groups;
   if (*dev == nullptr)
     if (int r = dev_alloc(c, dev, (size_t)5 * g.n_layers + 1)) return r;
   CU_OK(c, cudaMemcpyAsync(*dev, prog.data(), prog.size() * sizeof(StageDesc), cudaMemcpyHostToDevice, c->stream));
@@ -292,7 +302,7 @@ int build_programs(sdfp_ctx* c) {
 
 template <int CG, int HD>
 size_t pass_smem_bytes(int n_slots) {
-  return (size_t)n_slots * kSlotBytes + pass_work_bytes<CG, HD>() + sizeof(PassShared);
+  return (size_t)n_slots * kSlotBytes + pass_work_bytes<HD>() + sizeof(PassShared);
 }
 
 // Largest ring that fits beside the work area of the widest instantiation (two column groups).
@@ -331,22 +341,21 @@ cudaError_t launch_pass_t(sdfp_ctx* c, const PassParams& pp) {
   return cudaLaunchKernelEx(&lc, pass_kernel<CG, HD>, pp, c->pass_slots);
 }
 
-cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, int n_chunks, bool with_lm_head) {
+cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool with_lm_head) {
   PassParams pp{};
   pp.prog = draft ? c->prog_d : c->prog_t;
   pp.n_stages = (draft ? c->n_prog_d : c->n_prog_t) - (with_lm_head ? 0 : 1);
   pp.M = rows;
   pp.rows_per_seq = rows_per_seq;
-  pp.n_chunks = n_chunks;
   pp.row_pos = c->plan.row_pos;
   pp.row_seq = c->plan.row_seq;
   pp.eps = c->cfg.rms_eps;
   pp.attn_scale = 1.0f / std::sqrt((float)c->cfg.head_dim);
   pp.part_o = c->part_o;
   pp.part_ml = c->part_ml;
-  pp.attn_counters = c->attn_counters;
   pp.split_partials = c->split_partials;
   pp.split_flags = c->split_flags;
+  pp.ssq_part = c->ssq_part;
   pp.sync = c->psync;
   const bool hd128 = c->cfg.head_dim == 128;
   if (rows <= 8) return hd128 ? launch_pass_t<1, 128>(c, pp) : launch_pass_t<1, 64>(c, pp);
@@ -372,7 +381,7 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
                     reinterpret_cast<const float*>(c->embed), c->h, d));
   const KvCache& kv = draft ? c->cache_d : c->cache_t;
   const bool whole_pass = c->use_pass && rows <= kPassMaxRows;
-  if (whole_pass) CU_OK(c, run_pass(c, draft, rows, attn_rows_per_seq, n_chunks, decide != DECIDE_NONE));
+  if (whole_pass) CU_OK(c, run_pass(c, draft, rows, attn_rows_per_seq, decide != DECIDE_NONE));
   for (int l = 0; l < g.n_layers && !whole_pass; ++l) {
     if (draft && !c->keep[l]) continue;  // Algorithm 1: pruned layers are removed from the draft
     const LayerWeights& lw = c->layers[l];
@@ -600,7 +609,8 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
     return bail(SDFP_ECUDA);
   }
   c->num_sms = prop.multiProcessorCount;
-  c->use_pass = c->use_mma && !(g.flags & SDFP_FLAG_NO_PASS_KERNEL) && prop.cooperativeLaunch && g.d_model >= 64;
+  c->use_pass = c->use_mma && !(g.flags & SDFP_FLAG_NO_PASS_KERNEL) && prop.cooperativeLaunch && g.d_model >= 64 &&
+                g.n_heads <= kPassMaxHeads && g.d_model / 128 + 1 <= kSsqMaxGroups;
   if (c->use_pass) {
     int optin = 0;
     cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
@@ -638,7 +648,7 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
     }
   }
   const size_t R = kMaxRows;
-  c->n_chunks_cap = (g.max_seq + kAttnChunk - 1) / kAttnChunk;
+  c->n_chunks_cap = std::max(2, (g.max_seq + kAttnChunk - 1) / kAttnChunk);  // >= 16 rows x kAttnSplits partials
   c->stats_cap = g.max_seq;
   if ((r = dev_alloc(c, &c->h, R * g.d_model, true)) || (r = dev_alloc(c, &c->q, R * g.d_model, true)) ||
       (r = dev_alloc(c, &c->att, R * g.d_model, true)) || (r = dev_alloc(c, &c->u, R * g.d_ffn, true)) ||
@@ -659,7 +669,8 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   if (c->use_pass) {
     if ((r = dev_alloc(c, &c->psync, 1, true)) ||
         (r = dev_alloc(c, &c->split_partials, (size_t)c->pass_grid * kUnitTiles * 2 * 64 * 2, true)) ||
-        (r = dev_alloc(c, &c->split_flags, (size_t)c->pass_grid, true)) || (r = build_programs(c)))
+        (r = dev_alloc(c, &c->split_flags, (size_t)c->pass_grid, true)) ||
+        (r = dev_alloc(c, &c->ssq_part, (size_t)kSsqMaxGroups * kPassMaxRows, true)) || (r = build_programs(c)))
       return bail(r);
   }
   if (cudaMallocHost(reinterpret_cast<void**>(&c->pinned_flag), 64) != cudaSuccess) {
@@ -710,7 +721,6 @@ int check_pass_error(sdfp_ctx* c) {
   if (ps.error == 0) return 0;
   cudaMemsetAsync(c->psync, 0, sizeof(PassSync), c->stream);
   cudaMemsetAsync(c->split_flags, 0, (size_t)c->pass_grid * sizeof(unsigned), c->stream);
-  cudaMemsetAsync(c->attn_counters, 0, (size_t)kMaxRows * c->cfg.n_heads * sizeof(int), c->stream);
   cudaStreamSynchronize(c->stream);
   static const char* const what[] = {"", "grid barrier", "weight slot never filled", "weight slot never freed",
                                      "partial sum of a split group never posted"};
@@ -967,7 +977,8 @@ extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int3
   const int per_pass = std::min((int)rows, c->use_pass ? kPassMaxRows : kMaxRows);
   const int rps = std::min(per_pass, kAttnMaxR);
   const int prow = ((per_pass + rps - 1) / rps) * rps;
-  const int n_chunks = (start + rows + kAttnChunk - 1) / kAttnChunk;
+  // partials per (row, head): one per 64-key chunk, or a fixed kAttnSplits in the whole-pass kernel
+  const int n_chunks = c->use_pass ? kAttnSplits : (start + rows + kAttnChunk - 1) / kAttnChunk;
   // layout inside the array: arrival counters | (max, sum) partials | o partials
   const size_t counters_bytes = round_up_256((size_t)kMaxRows * g.n_heads * sizeof(int));
   const size_t ml_bytes = round_up_256((size_t)prow * g.n_heads * n_chunks * 2 * sizeof(float));
@@ -975,7 +986,7 @@ extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int3
   const size_t need = counters_bytes + ml_bytes + o_bytes;
   if (need > kStaticScratchBytes)
     return fail(c, SDFP_EINVAL,
-                "sdfp_forward_logits_static: %d rows x %d heads x %d key chunks need %zu bytes of attention scratch, "
+                "sdfp_forward_logits_static: %d rows x %d heads x %d partials need %zu bytes of attention scratch, "
                 "the static array holds %zu; use fewer rows per call, a shorter context, or sdfp_forward_logits",
                 prow, g.n_heads, n_chunks, need, kStaticScratchBytes);
   unsigned char* base = nullptr;

@@ -45,19 +45,26 @@ constexpr int kUnitTiles = 8;                            // row tiles per unit
 constexpr int kUnitBytes = kUnitTiles * 512;
 constexpr int kChunkUnits = 4;  // units per ring slot = number of k-classes
 constexpr int kSlotBytes = kChunkUnits * kUnitBytes;
-constexpr int kPassMaxRows = 16;  // rows one launch may carry (two column groups of 8)
-constexpr int kPassAttnR = 16;    // rows of one sequence per attention item
+constexpr int kPassMaxRows = 16;   // rows one launch may carry (two column groups of 8)
+constexpr int kPassAttnR = 16;     // rows of one sequence per attention item
+constexpr int kAttnSplits = 8;     // a head's 64-key chunks are dealt round-robin to this many items
+constexpr int kSsqMaxGroups = 256;  // groups of 128 features of the residual stream (d_model <= 32768)
 
 enum StageKind { ST_LINEAR = 0, ST_ATTN = 1 };
+enum XMode { X_PLAIN = 0, X_ATTN_FOLD = 1 };          // how a linear stage reads its activations
+enum RmsMode { RMS_NONE = 0, RMS_DIRECT = 1, RMS_FROM_PARTS = 2 };
 
 struct StageDesc {
   int kind;
   int K, KT, NT, n_groups;  // linear: in-features, k-tiles, row tiles, groups of 8 row tiles
   int ldx;
+  int x_mode, rms_mode;
+  int write_ssq;      // EPI_RESID stages: leave per-group sums of squares of the new residual rows
+  int ssq_groups;     // RMS_FROM_PARTS: how many group sums make a row's sum
   const uint4* W;     // unit layout
   const float* X;     // linear: activations [rows, K]; attention: q [rows, d_model]
   const float* gain;  // linear: RMSNorm gain or null
-  EpiParams ep;       // linear epilogue; attention: out, kcache, vcache, n_heads, max_seq
+  EpiParams ep;       // linear epilogue; attention: kcache, vcache, n_heads, max_seq
 };
 
 // what a wait that gave up leaves in PassSync::error
@@ -65,9 +72,11 @@ enum PassError { PASS_OK = 0, PASS_ERR_GRID_BARRIER = 1, PASS_ERR_SLOT_FULL = 2,
 
 struct PassSync {       // one per context, in global memory, zero-initialised
   unsigned bar_count;   // grid-barrier arrivals, ever increasing (wraps)
-  unsigned bar_base;    // value of bar_count when the running launch started
-  unsigned epoch_base;  // serial number of the last stage of the previous launch
+  unsigned pad0[31];
+  unsigned bar_gen;     // target of the last barrier that completed; written by its last arriver
+  unsigned pad1[31];
   int error;            // first PassError seen, sticky
+  unsigned pad2[31];
 };
 
 struct PassParams {
@@ -75,17 +84,16 @@ struct PassParams {
   int n_stages;
   int M;             // rows in this pass (<= kPassMaxRows); rows beyond carry nothing
   int rows_per_seq;  // attention: rows m0..m0+R-1 of a group belong to one sequence
-  int n_chunks;      // attention: 64-key chunks that bound the context
   const int* row_pos;
   const int* row_seq;
   float eps;
   float attn_scale;
   // scratch
-  float* part_o;          // attention partials [rows][head][chunk][head_dim]
-  float* part_ml;         // [rows][head][chunk][2]
-  int* attn_counters;     // [groups][head], zero between launches
+  float* part_o;          // attention partials [rows][head][kAttnSplits][head_dim], not normalised
+  float* part_ml;         // [rows][head][kAttnSplits][2] running max and sum
   float* split_partials;  // [grid][kUnitTiles * CG * 64 * 2]
   unsigned* split_flags;  // [grid]
+  float* ssq_part;        // [kSsqMaxGroups][kPassMaxRows]
   PassSync* sync;
 };
 
@@ -125,8 +133,10 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
 __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ void red_release_add(unsigned* p, unsigned v) {
-  asm volatile("red.release.gpu.global.add.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ unsigned atom_add_release(unsigned* p, unsigned v) {
+  unsigned old;
+  asm volatile("atom.add.release.gpu.global.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
+  return old;
 }
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
@@ -147,7 +157,7 @@ struct PassShared {
   int abort;     // set by whichever thread gives up a wait
   int decision;  // abort as sampled by thread 0 between two consumer barriers: uniform for all
   int attn_pos[2][kPassAttnR];
-  int attn_last[2];
+  float attn_m[2][kPassAttnR], attn_l[2][kPassAttnR], attn_a[2][kPassAttnR];
   int n_parts;
   int parts[160];  // CTAs that post a partial for the group this CTA finishes
 };
@@ -186,13 +196,19 @@ __device__ __forceinline__ bool bounded_wait(Pred pred, PassSync* sync, volatile
 }
 
 // ---- grid barrier (consumer threads of every CTA) ------------------------------------------------
-// Everything the consumer threads of this CTA wrote before is visible to every CTA after.
+// Everything the consumer threads of this CTA wrote before is visible to every CTA after.  The
+// arrivals go to one counter; the CTA that completes the count publishes the barrier's target in a
+// word of its own cache line, which is all the others poll, so polling never collides with arrivals.
 __device__ __forceinline__ bool grid_barrier(PassSync* sync, unsigned target, PassShared* sh) {
   consumer_sync();
   if (threadIdx.x == 0) {
     __threadfence();
-    red_release_add(&sync->bar_count, 1u);
-    bounded_wait([&] { return (int)(ld_acquire(&sync->bar_count) - target) >= 0; }, sync, &sh->abort, PASS_ERR_GRID_BARRIER);
+    const unsigned old = atom_add_release(&sync->bar_count, 1u);
+    if (old + 1u == target) {
+      st_release(&sync->bar_gen, target);
+    } else {
+      bounded_wait([&] { return (int)(ld_acquire(&sync->bar_gen) - target) >= 0; }, sync, &sh->abort, PASS_ERR_GRID_BARRIER);
+    }
     sh->decision = sh->abort;
   }
   consumer_sync();
@@ -207,34 +223,76 @@ __device__ __forceinline__ void unit_range(long long n_units, int cta, int n_cta
 // ---- one linear stage, consumer side -------------------------------------------------------------
 template <int CG>
 struct XRegs {
-  float2 lo8[CG], hi8[CG];
+  float2 lo8[CG], hi8[CG];  // x[m][16kt + 2q .. +1] and x[m][16kt + 2q + 8 .. +9], m = 8 cg + g
+  float2 g0, g1;            // the RMSNorm gain at the same columns (1 when the stage has no norm)
 };
 
-template <int CG>
-__device__ __forceinline__ void load_xregs(XRegs<CG>& x, const float* X, int ldx, int M, int kt, int g, int q, bool valid) {
+// Activation fragment of k-tile kt for every column group, with the gain at those columns.
+// X_ATTN_FOLD: the activation is the attention output, which exists only as kAttnSplits partial
+// sums per (row, head); sc[m][head - head0][j] holds exp(m_j - max)/sum for the heads this CTA
+// touches, and the fragment is the weighted sum of the partials in split order.
+template <int CG, int HD>
+__device__ __forceinline__ void load_xregs(XRegs<CG>& x, const StageDesc& st, const PassParams& pp, const float* sc, int head0,
+                                           int n_heads_local, int M, int kt, int g, int q, bool valid) {
+  x.g0 = make_float2(1.f, 1.f);
+  x.g1 = make_float2(1.f, 1.f);
+  if (valid && st.gain != nullptr) {
+    const float* gp = st.gain + kt * 16 + 2 * q;
+    x.g0 = *reinterpret_cast<const float2*>(gp);
+    x.g1 = *reinterpret_cast<const float2*>(gp + 8);
+  }
 #pragma unroll
   for (int cg = 0; cg < CG; ++cg) {
     const int m = cg * 8 + g;
     x.lo8[cg] = make_float2(0.f, 0.f);
     x.hi8[cg] = make_float2(0.f, 0.f);
     if (valid && m < M) {
-      const float* xp = X + (size_t)m * ldx + kt * 16 + 2 * q;
-      x.lo8[cg] = ld_act2(xp);
-      x.hi8[cg] = ld_act2(xp + 8);
+      if (st.x_mode == X_PLAIN) {
+        const float* xp = st.X + (size_t)m * st.ldx + kt * 16 + 2 * q;
+        x.lo8[cg] = ld_act2(xp);
+        x.hi8[cg] = ld_act2(xp + 8);
+      } else {
+        const int k = kt * 16 + 2 * q;
+        const int head = k / HD, d = k - head * HD;
+        const float* po = pp.part_o + (((size_t)m * st.ep.n_heads + head) * kAttnSplits) * HD + d;
+        const float* s8 = sc + ((size_t)m * n_heads_local + (head - head0)) * kAttnSplits;
+        float2 lo = make_float2(0.f, 0.f), hi = make_float2(0.f, 0.f);
+#pragma unroll
+        for (int j = 0; j < kAttnSplits; ++j) {
+          const float w = s8[j];
+          const float2 a = ld_act2(po + (size_t)j * HD);
+          const float2 b = ld_act2(po + (size_t)j * HD + 8);
+          lo.x = fmaf(w, a.x, lo.x);
+          lo.y = fmaf(w, a.y, lo.y);
+          hi.x = fmaf(w, b.x, hi.x);
+          hi.y = fmaf(w, b.y, hi.y);
+        }
+        x.lo8[cg] = lo;
+        x.hi8[cg] = hi;
+      }
     }
   }
 }
 
-template <int CG>
-__device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigned char* ring, int n_slots, float4* red,
+// work-area layout (bytes from its start)
+constexpr int kWorkRedBytes = 4 * kUnitTiles * 2 * 32 * 16;  // class partials, two column groups
+constexpr int kWorkSqOff = kWorkRedBytes;                    // squares of new residual values [it]
+constexpr int kWorkSqBytes = kUnitTiles * 2 * 64 * 4;
+constexpr int kWorkScOff = kWorkSqOff + kWorkSqBytes;        // attention fold weights
+constexpr int kPassMaxHeads = 48;
+constexpr int kWorkScBytes = kPassMaxRows * kPassMaxHeads * kAttnSplits * 4;
+
+template <int CG, int HD>
+__device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigned char* ring, int n_slots, unsigned char* work,
                              unsigned& chunk_base, unsigned epoch) {
   const StageDesc& st = sh->st;
+  float4* red = reinterpret_cast<float4*>(work);
+  float* sq_buf = reinterpret_cast<float*>(work + kWorkSqOff);
+  float* sc = reinterpret_cast<float*>(work + kWorkScOff);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, q = lane & 3;
   const int cls = warp & 3, th = warp >> 2;
-  const int KT = st.KT, M = pp.M, ldx = st.ldx;
-  const float* const X = st.X;
-  const float* const gain = st.gain;
+  const int KT = st.KT, M = pp.M;
   const int cta = blockIdx.x, n_cta = gridDim.x;
   const long long n_units = (long long)st.n_groups * KT;
   long long ub64, ue64;
@@ -245,11 +303,11 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   const int grp0 = (int)(ub64 / KT);
   const int kt_first = (int)(ub64 - (long long)grp0 * KT);  // k-tile of unit 0
 
-  // 1/rms of every row: the same fixed-order sum in every CTA
-  if (gain != nullptr) {
+  // ---- 1/rms of every row (needed only by the epilogue) ----
+  if (st.rms_mode == RMS_DIRECT) {
     float* s_part = reinterpret_cast<float*>(red);  // [warp][row]
     for (int m = 0; m < M; ++m) {
-      const float* x = X + (size_t)m * ldx;
+      const float* x = st.X + (size_t)m * st.ldx;
       float s = 0.f;
       for (int k = tid * 4; k < st.K; k += kPassConsumerThreads * 4) {
         const float4 v = ld_act4(x + k);
@@ -268,16 +326,43 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
       for (int w = 0; w < kPassConsumerWarps; ++w) s += s_part[w * kPassMaxRows + tid];
       sh->inv_rms[tid] = rsqrtf(s / (float)st.K + pp.eps);
     }
-  } else if (tid < kPassMaxRows) {
+    consumer_sync();
+  } else if (st.rms_mode == RMS_NONE && tid < kPassMaxRows) {
     sh->inv_rms[tid] = 1.f;
   }
-  consumer_sync();
+
+  // ---- attention fold weights: per (row, head) the factor of each split's partial ----
+  const int head0 = 0, n_heads_local = st.ep.n_heads;
+  if (st.x_mode == X_ATTN_FOLD) {
+    for (int e = tid; e < M * n_heads_local; e += kPassConsumerThreads) {
+      const float* ml = pp.part_ml + (size_t)e * kAttnSplits * 2;  // e = m * n_heads + head
+      float mj[kAttnSplits], lj[kAttnSplits];
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < kAttnSplits; ++j) {
+        const float2 v = ld_act2(ml + 2 * j);
+        mj[j] = v.x;
+        lj[j] = v.y;
+        if (v.y > 0.f) mx = fmaxf(mx, v.x);
+      }
+      float l = 0.f, wj[kAttnSplits];
+#pragma unroll
+      for (int j = 0; j < kAttnSplits; ++j) {
+        wj[j] = lj[j] > 0.f ? __expf(mj[j] - mx) : 0.f;
+        l = fmaf(lj[j], wj[j], l);
+      }
+      const float inv_l = l > 0.f ? 1.0f / l : 0.f;
+#pragma unroll
+      for (int j = 0; j < kAttnSplits; ++j) sc[(size_t)e * kAttnSplits + j] = wj[j] * inv_l;
+    }
+    consumer_sync();
+  }
 
   // activation fragments of my next four units; kt_pref = k-tile of the next unit to prefetch
   XRegs<CG> x0, x1, x2, x3;
   int kt_pref = (kt_first + cls) % KT;
   auto prefetch = [&](XRegs<CG>& x, int i) {
-    load_xregs<CG>(x, X, ldx, M, kt_pref, g, q, i < my_n);
+    load_xregs<CG, HD>(x, st, pp, sc, head0, n_heads_local, M, kt_pref, g, q, i < my_n);
     kt_pref += kChunkUnits;
     if (kt_pref >= KT) kt_pref -= KT;
   };
@@ -285,6 +370,13 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   prefetch(x1, 1);
   prefetch(x2, 2);
   prefetch(x3, 3);
+  if (st.rms_mode == RMS_FROM_PARTS && tid < M) {
+    // the stage that produced the residual stream left one sum of squares per 128-feature group;
+    // issued after the activation loads, read by the epilogue behind at least one barrier
+    float s = 0.f;
+    for (int gi = 0; gi < st.ssq_groups; ++gi) s += ld_act(pp.ssq_part + gi * kPassMaxRows + tid);
+    sh->inv_rms[tid] = rsqrtf(s / (float)st.K + pp.eps);
+  }
 
   int i = 0;          // my next unit is number cls + 4 i
   int seg_begin = 0;  // in units from ub64
@@ -293,6 +385,30 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   while (seg_begin < nun) {
     const int seg_len = min(nun - seg_begin, KT - seg_kt0);
     const int seg_end = seg_begin + seg_len;
+    const bool starts_group = (seg_kt0 == 0);
+    const bool whole = starts_group && (seg_len == KT);
+    const bool owner = starts_group && !whole;
+
+    // the old residual values this thread will add to, fetched now so that they are there at the end
+    float2 hold[2 * CG];
+#pragma unroll
+    for (int j = 0; j < 2 * CG; ++j) hold[j] = make_float2(0.f, 0.f);
+    if (starts_group && st.ep.mode == EPI_RESID) {
+#pragma unroll
+      for (int j = 0; j < 2 * CG; ++j) {
+        const int it = tid + j * kPassConsumerThreads;
+        const int ch = it & 1, ln = (it >> 1) & 31, rc = it >> 6;
+        const int cg = rc % CG, tile = rc / CG;
+        const int m = cg * 8 + 2 * (ln & 3) + ch;
+        const int rt = grp * kUnitTiles + tile;
+        hold[j] = make_float2(0.f, 0.f);
+        if (m < M && rt < st.NT) {
+          const float* hp = st.ep.out + (size_t)m * st.ep.out_ld + 16 * rt + (ln >> 2);
+          hold[j] = make_float2(ld_act(hp), ld_act(hp + 8));
+        }
+      }
+    }
+
     float acc[4][CG][4];
 #pragma unroll
     for (int r = 0; r < 4; ++r)
@@ -303,7 +419,6 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
 
     bool warp_ok = true;
     while (warp_ok && i < my_n && cls + kChunkUnits * i < seg_end) {
-      const int kt = seg_kt0 + (cls + kChunkUnits * i - seg_begin);
       const unsigned gc = chunk_base + (unsigned)i;
       const unsigned slot = gc % (unsigned)n_slots, parity = (gc / (unsigned)n_slots) & 1u;
       // Lanes leave the polling loop at different times.  mma.sync needs the whole warp
@@ -315,17 +430,11 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
       uint4 a[4];
 #pragma unroll
       for (int r = 0; r < 4; ++r) a[r] = tiles[r * 32 + lane];
-      float2 g0 = make_float2(1.f, 1.f), g1 = make_float2(1.f, 1.f);
-      if (gain != nullptr) {
-        const float* gp = gain + kt * 16 + 2 * q;
-        g0 = *reinterpret_cast<const float2*>(gp);
-        g1 = *reinterpret_cast<const float2*>(gp + 8);
-      }
 #pragma unroll
       for (int cg = 0; cg < CG; ++cg) {
         uint32_t bh0, bl0, bh1, bl1;
-        split_pack(x0.lo8[cg].x * g0.x, x0.lo8[cg].y * g0.y, bh0, bl0);
-        split_pack(x0.hi8[cg].x * g1.x, x0.hi8[cg].y * g1.y, bh1, bl1);
+        split_pack(x0.lo8[cg].x * x0.g0.x, x0.lo8[cg].y * x0.g0.y, bh0, bl0);
+        split_pack(x0.hi8[cg].x * x0.g1.x, x0.hi8[cg].y * x0.g1.y, bh1, bl1);
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
           mma_bf16_16816(acc[r][cg], a[r], bh0, bh1);
@@ -353,30 +462,34 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
       for (int cg = 0; cg < CG; ++cg)
         red[((cls * kUnitTiles + th * 4 + r) * CG + cg) * 32 + lane] =
             make_float4(acc[r][cg][0], acc[r][cg][1], acc[r][cg][2], acc[r][cg][3]);
-    const bool starts_group = (seg_kt0 == 0);
-    const bool whole = starts_group && (seg_len == KT);
-    const bool owner = starts_group && !whole;
-    if (owner && tid == 0) {
-      // the rest of the group sits at the beginning of the ranges of the CTAs that follow
+    if (owner && warp == 0) {
+      // The rest of the group sits at the beginning of the ranges of the CTAs that follow; every
+      // lane looks at one candidate and waits for that CTA's flag, so the waits overlap.
       const long long grp_end = (long long)(grp + 1) * KT;
       int n = 0;
-      bool w_ok = true;
-      for (int c2 = cta + 1; c2 < n_cta && w_ok; ++c2) {
-        long long b2, e2;
-        unit_range(n_units, c2, n_cta, b2, e2);
-        if (b2 >= grp_end) break;
-        if (e2 == b2) continue;  // an empty range posts nothing
-        sh->parts[n++] = c2;
-        w_ok = bounded_wait([&] { return ld_acquire(pp.split_flags + c2) == epoch; }, pp.sync, &sh->abort, PASS_ERR_SPLIT_FLAG);
+      bool more = true;
+      for (int base = cta + 1; more; base += 32) {
+        const int c2 = base + lane;
+        long long b2 = grp_end, e2 = grp_end;
+        if (c2 < n_cta) unit_range(n_units, c2, n_cta, b2, e2);
+        const bool beyond = (c2 >= n_cta) || (b2 >= grp_end);
+        const bool part = !beyond && e2 > b2;  // an empty range posts nothing
+        if (part) bounded_wait([&] { return ld_acquire(pp.split_flags + c2) == epoch; }, pp.sync, &sh->abort, PASS_ERR_SPLIT_FLAG);
+        const unsigned mask = __ballot_sync(0xffffffffu, part);
+        if (part) sh->parts[n + __popc(mask & ((1u << lane) - 1u))] = c2;
+        n += __popc(mask);
+        more = !__any_sync(0xffffffffu, beyond);
       }
-      sh->n_parts = n;
+      if (lane == 0) sh->n_parts = n;
     }
     if (!consumers_agree_ok(sh)) return;
 
     {
       float2* my_post = reinterpret_cast<float2*>(pp.split_partials) + (size_t)cta * (kUnitTiles * CG * 64);
       const int n_parts = owner ? sh->n_parts : 0;
-      for (int it = tid; it < kUnitTiles * CG * 64; it += kPassConsumerThreads) {
+#pragma unroll
+      for (int j = 0; j < 2 * CG; ++j) {
+        const int it = tid + j * kPassConsumerThreads;
         const int ch = it & 1;
         const int ln = (it >> 1) & 31;
         const int rc = it >> 6;
@@ -392,18 +505,39 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
           my_post[it] = make_float2(v0, v1);
           continue;
         }
-        for (int j = 0; j < n_parts; ++j) {
+        for (int k2 = 0; k2 < n_parts; ++k2) {
           const float2 o =
-              __ldcg(reinterpret_cast<const float2*>(pp.split_partials) + (size_t)sh->parts[j] * (kUnitTiles * CG * 64) + it);
+              __ldcg(reinterpret_cast<const float2*>(pp.split_partials) + (size_t)sh->parts[k2] * (kUnitTiles * CG * 64) + it);
           v0 += o.x;
           v1 += o.y;
         }
         const int m = cg * 8 + 2 * (ln & 3) + ch;
         const int rt = grp * kUnitTiles + tile;
+        float sq = 0.f;
         if (m < M && rt < st.NT) {
           const float inv = sh->inv_rms[m];
-          apply_epilogue<__nv_bfloat16>(st.ep, 8 * rt + (ln >> 2), m, v0 * inv, v1 * inv);
+          if (st.ep.mode == EPI_RESID) {
+            float* hp = st.ep.out + (size_t)m * st.ep.out_ld + 16 * rt + (ln >> 2);
+            const float n0 = hold[j].x + v0 * inv, n1 = hold[j].y + v1 * inv;
+            hp[0] = n0;
+            hp[8] = n1;
+            sq = fmaf(n0, n0, n1 * n1);
+          } else {
+            apply_epilogue<__nv_bfloat16>(st.ep, 8 * rt + (ln >> 2), m, v0 * inv, v1 * inv);
+          }
         }
+        if (st.write_ssq) sq_buf[it] = sq;
+      }
+    }
+    if (starts_group && st.write_ssq) {
+      // one sum of squares per row over this group's 128 features, in tile-then-row order
+      consumer_sync();
+      if (tid < M) {
+        const int cg = tid >> 3, qq = (tid & 7) >> 1, ch = tid & 1;
+        float s = 0.f;
+        for (int tile = 0; tile < kUnitTiles; ++tile)
+          for (int g8 = 0; g8 < 8; ++g8) s += sq_buf[(((tile * CG + cg) * 32) + g8 * 4 + qq) * 2 + ch];
+        pp.ssq_part[grp * kPassMaxRows + tid] = s;
       }
     }
     if (!starts_group) __threadfence();  // every thread publishes its own part of the partial sum
@@ -430,36 +564,57 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   chunk_base += (unsigned)n_chunks;
 }
 
-// ---- attention stage: one item = (64-key chunk, head, row group), handled by half a CTA -------------
+// ---- attention stage --------------------------------------------------------------------------
+// One item = (head, split j, row group), handled by half a CTA.  Split j owns the 64-key chunks
+// j, j + kAttnSplits, ... of the head (chunk grid fixed in absolute key index) and walks them in
+// order with a running max and sum per row; it leaves an un-normalised partial (max, sum, o) per
+// row.  The O-projection that follows combines the kAttnSplits partials in split order while it
+// loads its activations, so nothing waits on another CTA inside this stage.  A row's numbers
+// depend only on its own position: rows that cannot see a chunk skip it entirely.
 template <int HD>
 __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassShared* sh, unsigned char* smem, int half,
-                               int htid, int c, int head, int b) {
+                               int htid, int head, int split, int b) {
   using KT = __nv_bfloat16;
   constexpr int C = kAttnChunk;
   KT* sV = reinterpret_cast<KT*>(smem);               // [C][HD]
   float* sQ = reinterpret_cast<float*>(sV + C * HD);  // [R][HD]
   float* sS = sQ + kPassAttnR * HD;                   // [R][C]
   int* s_pos = sh->attn_pos[half];
+  float* s_m = sh->attn_m[half];
+  float* s_l = sh->attn_l[half];
+  float* s_a = sh->attn_a[half];
   const int R = pp.rows_per_seq;
   const int row0 = b * R;
-  const int key0 = c * C;
   const int n_heads = st.ep.n_heads;
   const size_t d_model = (size_t)n_heads * HD;
 
-  if (htid < R) s_pos[htid] = (row0 + htid < pp.M) ? ld_act(pp.row_pos + row0 + htid) : -1;
+  if (htid < R) {
+    s_pos[htid] = (row0 + htid < pp.M) ? ld_act(pp.row_pos + row0 + htid) : -1;
+    s_m[htid] = -INFINITY;
+    s_l[htid] = 0.f;
+  }
   half_sync(half);
   int max_pos = -1;
   for (int i = 0; i < R; ++i) max_pos = max(max_pos, s_pos[i]);
+  const int seq = ld_act(pp.row_seq + row0);
+  for (int e = htid; e < R * HD; e += 128) {
+    const int i = e / HD, d = e - i * HD;
+    sQ[e] = (s_pos[i] >= 0) ? ld_act(st.X + (size_t)(row0 + i) * d_model + head * HD + d) : 0.f;
+  }
 
-  if (max_pos >= key0) {
-    const int seq = ld_act(pp.row_seq + row0);
+  float o[kPassAttnR];  // thread d < HD: o[i][d]
+#pragma unroll
+  for (int i = 0; i < kPassAttnR; ++i) o[i] = 0.f;
+
+  constexpr int KV4 = HD / 16;  // uint4 per half key row
+  constexpr int VPR = HD / 8;
+  const int key = htid >> 1, hf = htid & 1;
+  for (int c = split; c * C <= max_pos; c += kAttnSplits) {
+    const int key0 = c * C;
     const int nk_all = min(C, max_pos + 1 - key0);
     const size_t base = (((size_t)seq * n_heads + head) * st.ep.max_seq + key0) * HD;
     const KT* gK = reinterpret_cast<const KT*>(st.ep.kcache) + base;
     const KT* gV = reinterpret_cast<const KT*>(st.ep.vcache) + base;
-    // this thread's half of one key row goes straight to registers
-    constexpr int KV4 = HD / 16;  // uint4 per half row
-    const int key = htid >> 1, hf = htid & 1;
     uint4 kreg[KV4];
 #pragma unroll
     for (int j = 0; j < KV4; ++j) kreg[j] = make_uint4(0u, 0u, 0u, 0u);
@@ -468,15 +623,9 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
 #pragma unroll
       for (int j = 0; j < KV4; ++j) kreg[j] = __ldcg(kp + j);
     }
-    constexpr int VPR = HD / 8;
+    half_sync(half);  // the previous chunk's sV and sS are no longer read (and sQ is complete)
     for (int v = htid; v < nk_all * VPR; v += 128)
       reinterpret_cast<uint4*>(sV)[v] = __ldcg(reinterpret_cast<const uint4*>(gV) + v);
-    for (int e = htid; e < R * HD; e += 128) {
-      const int i = e / HD, d = e - i * HD;
-      sQ[e] = (s_pos[i] >= 0) ? ld_act(st.X + (size_t)(row0 + i) * d_model + head * HD + d) : 0.f;
-    }
-    half_sync(half);
-
     {
       float acc[kPassAttnR];
 #pragma unroll
@@ -508,80 +657,59 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
       }
     }
     half_sync(half);
-
     {
       const int w4 = htid >> 5, lane = htid & 31;
       for (int i = w4; i < R; i += 4) {
         const int nk = min(C, s_pos[i] + 1 - key0);
+        if (nk <= 0) {  // the row cannot see this chunk: leave its state alone
+          if (lane == 0) s_a[i] = 1.f;
+          sS[i * C + lane] = 0.f;
+          sS[i * C + lane + 32] = 0.f;
+          continue;
+        }
         const float s0 = (lane < nk) ? sS[i * C + lane] : -INFINITY;
         const float s1 = (lane + 32 < nk) ? sS[i * C + lane + 32] : -INFINITY;
-        const float mx = warp_max(fmaxf(s0, s1));
-        const float p0 = (lane < nk) ? __expf(s0 - mx) : 0.f;
-        const float p1 = (lane + 32 < nk) ? __expf(s1 - mx) : 0.f;
+        const float m_old = s_m[i];
+        const float m_new = fmaxf(m_old, warp_max(fmaxf(s0, s1)));
+        const float p0 = (lane < nk) ? __expf(s0 - m_new) : 0.f;
+        const float p1 = (lane + 32 < nk) ? __expf(s1 - m_new) : 0.f;
         sS[i * C + lane] = p0;
         sS[i * C + lane + 32] = p1;
-        const float l = warp_sum(p0 + p1);
-        if (lane == 0 && nk > 0) {
-          float* ml = pp.part_ml + ((((size_t)(row0 + i)) * n_heads + head) * pp.n_chunks + c) * 2;
-          ml[0] = mx;
-          ml[1] = l;
+        const float psum = warp_sum(p0 + p1);
+        if (lane == 0) {
+          const float alpha = __expf(m_old - m_new);  // exp(-inf) = 0 on the row's first chunk
+          s_a[i] = alpha;
+          s_m[i] = m_new;
+          s_l[i] = fmaf(s_l[i], alpha, psum);
         }
       }
     }
     half_sync(half);
-
-    for (int d = htid; d < HD; d += 128) {
-      float o[kPassAttnR];
+    if (htid < HD) {
 #pragma unroll
-      for (int i = 0; i < kPassAttnR; ++i) o[i] = 0.f;
+      for (int i = 0; i < kPassAttnR; ++i)
+        if (i < R) o[i] *= s_a[i];
       for (int k2 = 0; k2 < nk_all; ++k2) {
-        const float v = __bfloat162float(sV[k2 * HD + d]);
+        const float v = __bfloat162float(sV[k2 * HD + htid]);
 #pragma unroll
         for (int i = 0; i < kPassAttnR; ++i)
           if (i < R) o[i] = fmaf(sS[i * C + k2], v, o[i]);
       }
+    }
+  }
+  // the partial of every row of the group, also of rows that saw nothing here (sum 0)
+  if (htid < HD) {
 #pragma unroll
-      for (int i = 0; i < kPassAttnR; ++i)
-        if (i < R && s_pos[i] >= key0)
-          pp.part_o[((((size_t)(row0 + i)) * n_heads + head) * pp.n_chunks + c) * HD + d] = o[i];
-    }
+    for (int i = 0; i < kPassAttnR; ++i)
+      if (i < R && row0 + i < pp.M)
+        pp.part_o[((((size_t)(row0 + i)) * n_heads + head) * kAttnSplits + split) * HD + htid] = o[i];
   }
-
-  // the half-CTA that arrives last for this (group, head) folds the chunks in chunk order
-  __threadfence();
-  half_sync(half);
-  if (htid == 0) {
-    const int prev = atomicAdd(&pp.attn_counters[b * n_heads + head], 1);
-    sh->attn_last[half] = (prev == pp.n_chunks - 1);
+  if (htid < R && row0 + htid < pp.M) {
+    float* ml = pp.part_ml + ((((size_t)(row0 + htid)) * n_heads + head) * kAttnSplits + split) * 2;
+    ml[0] = s_m[htid];
+    ml[1] = s_l[htid];
   }
-  half_sync(half);
-  if (sh->attn_last[half]) {
-    __threadfence();
-    if (htid == 0) pp.attn_counters[b * n_heads + head] = 0;
-    for (int i = 0; i < R; ++i) {
-      if (row0 + i >= pp.M) break;
-      const int pos = s_pos[i];
-      float* dst = st.ep.out + (size_t)(row0 + i) * d_model + head * HD;
-      if (pos < 0) {
-        for (int d = htid; d < HD; d += 128) dst[d] = 0.f;
-        continue;
-      }
-      const int nc = pos / C + 1;
-      const float* ml = pp.part_ml + (((size_t)(row0 + i)) * n_heads + head) * pp.n_chunks * 2;
-      const float* po = pp.part_o + (((size_t)(row0 + i)) * n_heads + head) * pp.n_chunks * HD;
-      float mx = -INFINITY;
-      for (int cc = 0; cc < nc; ++cc) mx = fmaxf(mx, __ldcg(ml + cc * 2));
-      float l = 0.f;
-      for (int cc = 0; cc < nc; ++cc) l = fmaf(__ldcg(ml + cc * 2 + 1), __expf(__ldcg(ml + cc * 2) - mx), l);
-      const float inv_l = 1.0f / l;
-      for (int d = htid; d < HD; d += 128) {
-        float o = 0.f;
-        for (int cc = 0; cc < nc; ++cc) o = fmaf(__ldcg(po + (size_t)cc * HD + d), __expf(__ldcg(ml + cc * 2) - mx), o);
-        dst[d] = o * inv_l;
-      }
-    }
-  }
-  half_sync(half);  // smem and s_pos are reused by the next item
+  half_sync(half);  // smem and the per-row state are reused by the next item
 }
 
 template <int HD>
@@ -589,23 +717,19 @@ __host__ __device__ constexpr size_t pass_attn_smem_half() {
   return (size_t)kAttnChunk * HD * 2 + (size_t)kPassAttnR * HD * 4 + (size_t)kPassAttnR * kAttnChunk * 4;
 }
 
-template <int CG>
-__host__ __device__ constexpr size_t pass_red_bytes() {
-  return (size_t)4 * kUnitTiles * CG * 32 * sizeof(float4);
-}
-
-template <int CG, int HD>
+template <int HD>
 __host__ __device__ constexpr size_t pass_work_bytes() {
-  return pass_red_bytes<CG>() > 2 * pass_attn_smem_half<HD>() ? pass_red_bytes<CG>() : 2 * pass_attn_smem_half<HD>();
+  return (size_t)(kWorkScOff + kWorkScBytes) > 2 * pass_attn_smem_half<HD>() ? (size_t)(kWorkScOff + kWorkScBytes)
+                                                                              : 2 * pass_attn_smem_half<HD>();
 }
 
-// Dynamic shared memory: [ring: n_slots * 16 KB][work area: reduction buffer / attention tiles][PassShared]
+// Dynamic shared memory: [ring: n_slots * 16 KB][work area][PassShared]
 template <int CG, int HD>
 __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, int n_slots) {
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* ring = smem;
   unsigned char* work = smem + (size_t)n_slots * kSlotBytes;
-  PassShared* sh = reinterpret_cast<PassShared*>(work + pass_work_bytes<CG, HD>());
+  PassShared* sh = reinterpret_cast<PassShared*>(work + pass_work_bytes<HD>());
   const int tid = threadIdx.x;
 
   if (tid == 0) {
@@ -656,10 +780,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
   }
 
   // ================= consumer warps =================
-  const unsigned bar_base = *reinterpret_cast<volatile unsigned*>(&pp.sync->bar_base);
-  const unsigned epoch_base = *reinterpret_cast<volatile unsigned*>(&pp.sync->epoch_base);
+  // The last barrier of the previous launch left its target in bar_gen, and nothing changes it
+  // before every CTA of this launch has arrived at the first barrier, i.e. has read it here.
+  const unsigned bar_base = *reinterpret_cast<volatile unsigned*>(&pp.sync->bar_gen);
   unsigned chunk_base = 0;
-  float4* red = reinterpret_cast<float4*>(work);
   bool ok = true;
   for (int s = 0; s < pp.n_stages && ok; ++s) {
     {
@@ -669,27 +793,22 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
       consumer_sync();
     }
     if (sh->st.kind == ST_LINEAR) {
-      linear_stage<CG>(pp, sh, ring, n_slots, red, chunk_base, epoch_base + (unsigned)s + 1u);
+      // serial number of the stage over all launches: the posts of split groups carry it
+      linear_stage<CG, HD>(pp, sh, ring, n_slots, work, chunk_base, bar_base + (unsigned)s + 1u);
     } else {
       const int half = tid >> 7, htid = tid & 127;
       const int n_heads = sh->st.ep.n_heads;
       const int n_groups = (pp.M + pp.rows_per_seq - 1) / pp.rows_per_seq;
-      const int items = pp.n_chunks * n_heads * n_groups;
+      const int items = kAttnSplits * n_heads * n_groups;
       unsigned char* my = work + (size_t)half * pass_attn_smem_half<HD>();
       for (int it = blockIdx.x * 2 + half; it < items; it += gridDim.x * 2) {
-        const int c = it % pp.n_chunks;
-        const int hb = it / pp.n_chunks;
-        attention_item<HD>(sh->st, pp, sh, my, half, htid, c, hb % n_heads, hb / n_heads);
+        const int split = it % kAttnSplits;
+        const int hb = it / kAttnSplits;
+        attention_item<HD>(sh->st, pp, sh, my, half, htid, hb % n_heads, split, hb / n_heads);
       }
     }
     ok = consumers_agree_ok(sh);
     if (ok && s + 1 < pp.n_stages) ok = grid_barrier(pp.sync, bar_base + (unsigned)(s + 1) * gridDim.x, sh);
-  }
-  // the next launch starts from where this one ended (written after the last barrier, read by
-  // every CTA before its first one)
-  if (blockIdx.x == 0 && tid == 0 && ok) {
-    pp.sync->bar_base = bar_base + (unsigned)(pp.n_stages - 1) * gridDim.x;
-    pp.sync->epoch_base = epoch_base + (unsigned)pp.n_stages;
   }
 }
 

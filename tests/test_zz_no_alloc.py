@@ -49,12 +49,12 @@ def test_static_scratch_forward_matches_regular_forward(shape, tol):
 
 
 def test_static_scratch_rejects_what_does_not_fit():
-    """Even the narrowest pass of a 64-row call on 32 heads of width 128 needs about 266 KB of
-    partials per 64-key chunk: at a context of 2164 tokens (34 chunks) that is beyond the 8 MiB
-    array and must be refused with both sizes in the message, while a small call on the same
-    context is served."""
+    """With one kernel per operation, a 64-row call on 32 heads of width 128 needs about 1 MiB of
+    partials per 64-key chunk: at a context of 2164 tokens (34 chunks) that is far beyond the
+    8 MiB array and must be refused with both sizes in the message, while a small call on the
+    same context is served."""
     shape = si.LLAMA7B_4L
-    eng, m, _ = make_pair(shape, (1, 2), max_seq=2200, draw_device="cuda:0")
+    eng, m, _ = make_pair(shape, (1, 2), max_seq=2200, flags=pkg.FLAG_NO_PASS_KERNEL, draw_device="cuda:0")
     try:
         toks = si.make_prompts(shape.vocab, 1, 64, seed=22)[0].tolist()
         with pytest.raises(pkg.SdfpError) as ei:
