@@ -98,7 +98,7 @@ struct sdfp_ctx {
   float* split_partials = nullptr;
   unsigned* split_flags = nullptr;
   float* ssq_part = nullptr;
-  int pass_slots = 0;
+  int pass_slots[3] = {0, 0, 0};  // ring slots of the instantiation with 1 and with 2 column groups
   size_t pass_smem = 0;
   int pass_grid = 0;
   bool own_stream = false;
@@ -302,16 +302,23 @@ int build_programs(sdfp_ctx* c) {
 
 template <int CG, int HD>
 size_t pass_smem_bytes(int n_slots) {
-  return (size_t)n_slots * kSlotBytes + pass_work_bytes<HD>() + sizeof(PassShared);
+  return (size_t)n_slots * kSlotBytes + pass_work_bytes<CG, HD>() + sizeof(PassShared);
 }
 
-// Largest ring that fits beside the work area of the widest instantiation (two column groups).
+template <int CG, int HD>
+int pass_slots_that_fit(int max_smem_optin) {
+  int n_slots = 8;
+  while (n_slots > 2 && pass_smem_bytes<CG, HD>(n_slots) > (size_t)max_smem_optin) --n_slots;
+  return n_slots;
+}
+
+// Each instantiation gets the largest ring that fits beside its work area.
 template <int HD>
 cudaError_t configure_pass_t(sdfp_ctx* c, int max_smem_optin) {
-  int n_slots = 16;
-  while (n_slots > 2 && pass_smem_bytes<2, HD>(n_slots) > (size_t)max_smem_optin) --n_slots;
-  c->pass_slots = n_slots;
-  c->pass_smem = pass_smem_bytes<2, HD>(n_slots);
+  c->pass_slots[1] = pass_slots_that_fit<1, HD>(max_smem_optin);
+  c->pass_slots[2] = pass_slots_that_fit<2, HD>(max_smem_optin);
+  c->pass_smem = std::max(pass_smem_bytes<1, HD>(c->pass_slots[1]), pass_smem_bytes<2, HD>(c->pass_slots[2]));
+  if (c->pass_smem > (size_t)max_smem_optin) return cudaErrorLaunchOutOfResources;
   cudaError_t e = cudaFuncSetAttribute(pass_kernel<1, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_smem);
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(pass_kernel<2, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_smem);
@@ -338,7 +345,7 @@ cudaError_t launch_pass_t(sdfp_ctx* c, const PassParams& pp) {
   lc.attrs = attr;
   lc.numAttrs = 1;
   c->launches += 1;
-  return cudaLaunchKernelEx(&lc, pass_kernel<CG, HD>, pp, c->pass_slots);
+  return cudaLaunchKernelEx(&lc, pass_kernel<CG, HD>, pp, c->pass_slots[CG]);
 }
 
 cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool with_lm_head) {

@@ -11,7 +11,7 @@
 //     (cp.async.bulk + mbarrier transaction counts).  Weights do not depend on activations, so the
 //     producer runs ahead of the consumers across stage boundaries, through the grid barriers,
 //     as far as the ring allows (160 KB per SM, ~24 MB over the GPU).
-//   * Eight consumer warps take the slots in order, feed the tiles to mma.sync.m16n8k16 (weights
+//   * Sixteen consumer warps take the slots in order, feed the tiles to mma.sync.m16n8k16 (weights
 //     are the A operand, tokens the 8-wide B operand) and run the fused epilogues.
 //   * Stages are separated by a grid barrier (arrival counter in global memory, bounded spin).
 //
@@ -25,9 +25,9 @@
 // after the others have posted their partial sums to global scratch; partials are added in CTA
 // order, so the result does not depend on timing.
 //
-// Inside a CTA the 8 consumer warps are 4 k-classes x 2 tile halves: the unit with index
-// (range start + c + 4i) belongs to class c, and warp (c, t) multiplies its tiles 4t..4t+3.  The
-// four class partials are added in class order through shared memory.  All of this is fixed by
+// Inside a CTA the 16 consumer warps are 8 k-classes x 2 tile halves: the unit with index
+// (range start + c + 8i) belongs to class c, and warp (c, t) multiplies its tiles 4t..4t+3.  The
+// eight class partials are added in class order through shared memory.  All of this is fixed by
 // the matrix shape and the grid size alone, never by the number of rows, so a row's result is
 // bit-identical whether it is computed alone (autoregressive step) or among k+1 rows (verify).
 #pragma once
@@ -38,20 +38,23 @@
 
 namespace sdfp {
 
-constexpr int kPassConsumerWarps = 8;
+constexpr int kClasses = 8;  // k-classes: units of a CTA's range are dealt round-robin to them
+constexpr int kPassConsumerWarps = 2 * kClasses;
 constexpr int kPassConsumerThreads = kPassConsumerWarps * 32;
 constexpr int kPassThreads = kPassConsumerThreads + 32;  // + the producer warp
+constexpr int kHalfThreads = kPassConsumerThreads / 2;   // an attention item is run by half the consumers
 constexpr int kUnitTiles = 8;                            // row tiles per unit
 constexpr int kUnitBytes = kUnitTiles * 512;
-constexpr int kChunkUnits = 4;  // units per ring slot = number of k-classes
+constexpr int kChunkUnits = kClasses;  // units per ring slot
 constexpr int kSlotBytes = kChunkUnits * kUnitBytes;
-constexpr int kPassMaxRows = 16;   // rows one launch may carry (two column groups of 8)
-constexpr int kPassAttnR = 16;     // rows of one sequence per attention item
-constexpr int kAttnSplits = 8;     // a head's 64-key chunks are dealt round-robin to this many items
+constexpr int kPassMaxRows = 16;    // rows one launch may carry (two column groups of 8)
+constexpr int kPassAttnR = 16;      // rows of one sequence per attention item
+constexpr int kAttnSplits = 8;      // a head's 64-key chunks are dealt round-robin to this many items
+constexpr int kPassMaxHeads = 48;
 constexpr int kSsqMaxGroups = 256;  // groups of 128 features of the residual stream (d_model <= 32768)
 
 enum StageKind { ST_LINEAR = 0, ST_ATTN = 1 };
-enum XMode { X_PLAIN = 0, X_ATTN_FOLD = 1 };          // how a linear stage reads its activations
+enum XMode { X_PLAIN = 0, X_ATTN_FOLD = 1 };  // how a linear stage reads its activations
 enum RmsMode { RMS_NONE = 0, RMS_DIRECT = 1, RMS_FROM_PARTS = 2 };
 
 struct StageDesc {
@@ -70,12 +73,12 @@ struct StageDesc {
 // what a wait that gave up leaves in PassSync::error
 enum PassError { PASS_OK = 0, PASS_ERR_GRID_BARRIER = 1, PASS_ERR_SLOT_FULL = 2, PASS_ERR_SLOT_EMPTY = 3, PASS_ERR_SPLIT_FLAG = 4 };
 
-struct PassSync {       // one per context, in global memory, zero-initialised
-  unsigned bar_count;   // grid-barrier arrivals, ever increasing (wraps)
+struct PassSync {      // one per context, in global memory, zero-initialised
+  unsigned bar_count;  // grid-barrier arrivals, ever increasing (wraps)
   unsigned pad0[31];
-  unsigned bar_gen;     // target of the last barrier that completed; written by its last arriver
+  unsigned bar_gen;    // target of the last barrier that completed; written by its last arriver
   unsigned pad1[31];
-  int error;            // first PassError seen, sticky
+  int error;           // first PassError seen, sticky
   unsigned pad2[31];
 };
 
@@ -125,6 +128,11 @@ __device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned b
                "l"(src), "r"(bytes), "r"(smem_u32(bar))
                : "memory");
 }
+// 16-byte asynchronous copy global -> shared through L2 only (attention's V tiles)
+__device__ __forceinline__ void cp_async16(void* dst, const void* src) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
 __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
   unsigned v;
   asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
@@ -144,19 +152,19 @@ __device__ __forceinline__ unsigned long long global_ns() {
   return t;
 }
 __device__ __forceinline__ void consumer_sync() { asm volatile("bar.sync 1, %0;" ::"n"(kPassConsumerThreads) : "memory"); }
-__device__ __forceinline__ void half_sync(int half) { asm volatile("bar.sync %0, 128;" ::"r"(2 + half) : "memory"); }
+__device__ __forceinline__ void half_sync(int half) { asm volatile("bar.sync %0, %1;" ::"r"(2 + half), "n"(kHalfThreads) : "memory"); }
 
 // Every wait in this kernel gives up after this long, records why, and the kernel winds down.
 constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct PassShared {
-  uint64_t full[16];
-  uint64_t empty[16];
+  uint64_t full[8];
+  uint64_t empty[8];
   StageDesc st;  // the running stage, copied once per stage by the consumer threads
   float inv_rms[kPassMaxRows];
+  int row_pos[kPassMaxRows], row_seq[kPassMaxRows];  // fixed for the whole pass
   int abort;     // set by whichever thread gives up a wait
   int decision;  // abort as sampled by thread 0 between two consumer barriers: uniform for all
-  int attn_pos[2][kPassAttnR];
   float attn_m[2][kPassAttnR], attn_l[2][kPassAttnR], attn_a[2][kPassAttnR];
   int n_parts;
   int parts[160];  // CTAs that post a partial for the group this CTA finishes
@@ -224,38 +232,36 @@ __device__ __forceinline__ void unit_range(long long n_units, int cta, int n_cta
 template <int CG>
 struct XRegs {
   float2 lo8[CG], hi8[CG];  // x[m][16kt + 2q .. +1] and x[m][16kt + 2q + 8 .. +9], m = 8 cg + g
-  float2 g0, g1;            // the RMSNorm gain at the same columns (1 when the stage has no norm)
 };
 
-// Activation fragment of k-tile kt for every column group, with the gain at those columns.
-// X_ATTN_FOLD: the activation is the attention output, which exists only as kAttnSplits partial
-// sums per (row, head); sc[m][head - head0][j] holds exp(m_j - max)/sum for the heads this CTA
-// touches, and the fragment is the weighted sum of the partials in split order.
-template <int CG, int HD>
-__device__ __forceinline__ void load_xregs(XRegs<CG>& x, const StageDesc& st, const PassParams& pp, const float* sc, int head0,
-                                           int n_heads_local, int M, int kt, int g, int q, bool valid) {
-  x.g0 = make_float2(1.f, 1.f);
-  x.g1 = make_float2(1.f, 1.f);
-  if (valid && st.gain != nullptr) {
-    const float* gp = st.gain + kt * 16 + 2 * q;
-    x.g0 = *reinterpret_cast<const float2*>(gp);
-    x.g1 = *reinterpret_cast<const float2*>(gp + 8);
-  }
+struct XSource {  // the fields of the stage an activation load needs, kept in registers
+  const float* X;
+  const float* gain;
+  const float* part_o;
+  int ldx, n_heads;
+};
+
+// Activation fragment of k-tile kt for every column group.  X_ATTN_FOLD: the activation is the
+// attention output, which exists only as kAttnSplits partial sums per (row, head); sc[m][head][j]
+// holds exp(m_j - max)/sum, and the fragment is the weighted sum of the partials in split order.
+template <int CG, int HD, int XM>
+__device__ __forceinline__ void load_xregs(XRegs<CG>& x, const XSource& xs, const float* sc, int M, int kt, int g, int q,
+                                           bool valid) {
 #pragma unroll
   for (int cg = 0; cg < CG; ++cg) {
     const int m = cg * 8 + g;
     x.lo8[cg] = make_float2(0.f, 0.f);
     x.hi8[cg] = make_float2(0.f, 0.f);
     if (valid && m < M) {
-      if (st.x_mode == X_PLAIN) {
-        const float* xp = st.X + (size_t)m * st.ldx + kt * 16 + 2 * q;
+      if (XM == X_PLAIN) {
+        const float* xp = xs.X + (size_t)m * xs.ldx + kt * 16 + 2 * q;
         x.lo8[cg] = ld_act2(xp);
         x.hi8[cg] = ld_act2(xp + 8);
       } else {
         const int k = kt * 16 + 2 * q;
         const int head = k / HD, d = k - head * HD;
-        const float* po = pp.part_o + (((size_t)m * st.ep.n_heads + head) * kAttnSplits) * HD + d;
-        const float* s8 = sc + ((size_t)m * n_heads_local + (head - head0)) * kAttnSplits;
+        const float* po = xs.part_o + (((size_t)m * xs.n_heads + head) * kAttnSplits) * HD + d;
+        const float* s8 = sc + ((size_t)m * xs.n_heads + head) * kAttnSplits;
         float2 lo = make_float2(0.f, 0.f), hi = make_float2(0.f, 0.f);
 #pragma unroll
         for (int j = 0; j < kAttnSplits; ++j) {
@@ -274,25 +280,27 @@ __device__ __forceinline__ void load_xregs(XRegs<CG>& x, const StageDesc& st, co
   }
 }
 
-// work-area layout (bytes from its start)
-constexpr int kWorkRedBytes = 4 * kUnitTiles * 2 * 32 * 16;  // class partials, two column groups
-constexpr int kWorkSqOff = kWorkRedBytes;                    // squares of new residual values [it]
-constexpr int kWorkSqBytes = kUnitTiles * 2 * 64 * 4;
-constexpr int kWorkScOff = kWorkSqOff + kWorkSqBytes;        // attention fold weights
-constexpr int kPassMaxHeads = 48;
+// work-area layout of a linear stage (bytes from the start of the area)
+template <int CG>
+__host__ __device__ constexpr int work_red_bytes() { return kClasses * kUnitTiles * CG * 32 * 16; }  // class partials
+template <int CG>
+__host__ __device__ constexpr int work_sq_off() { return work_red_bytes<CG>(); }  // squares of new residual values [it]
+template <int CG>
+__host__ __device__ constexpr int work_sc_off() { return work_sq_off<CG>() + kUnitTiles * CG * 64 * 4; }  // attention fold weights
 constexpr int kWorkScBytes = kPassMaxRows * kPassMaxHeads * kAttnSplits * 4;
 
-template <int CG, int HD>
+template <int CG, int HD, int XM>
 __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigned char* ring, int n_slots, unsigned char* work,
                              unsigned& chunk_base, unsigned epoch) {
   const StageDesc& st = sh->st;
   float4* red = reinterpret_cast<float4*>(work);
-  float* sq_buf = reinterpret_cast<float*>(work + kWorkSqOff);
-  float* sc = reinterpret_cast<float*>(work + kWorkScOff);
+  float* sq_buf = reinterpret_cast<float*>(work + work_sq_off<CG>());
+  float* sc = reinterpret_cast<float*>(work + work_sc_off<CG>());
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, q = lane & 3;
-  const int cls = warp & 3, th = warp >> 2;
-  const int KT = st.KT, M = pp.M;
+  const int cls = warp & (kClasses - 1), th = warp / kClasses;
+  const int KT = st.KT, M = pp.M, NT = st.NT;
+  const int epi_mode = st.ep.mode;
   const int cta = blockIdx.x, n_cta = gridDim.x;
   const long long n_units = (long long)st.n_groups * KT;
   long long ub64, ue64;
@@ -302,6 +310,8 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   const int my_n = nun > cls ? (nun - cls + kChunkUnits - 1) / kChunkUnits : 0;
   const int grp0 = (int)(ub64 / KT);
   const int kt_first = (int)(ub64 - (long long)grp0 * KT);  // k-tile of unit 0
+  // ring position of this stage's first chunk; advanced by one slot per unit of this warp
+  unsigned slot = chunk_base % (unsigned)n_slots, parity = (chunk_base / (unsigned)n_slots) & 1u;
 
   // ---- 1/rms of every row (needed only by the epilogue) ----
   if (st.rms_mode == RMS_DIRECT) {
@@ -332,9 +342,9 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   }
 
   // ---- attention fold weights: per (row, head) the factor of each split's partial ----
-  const int head0 = 0, n_heads_local = st.ep.n_heads;
-  if (st.x_mode == X_ATTN_FOLD) {
-    for (int e = tid; e < M * n_heads_local; e += kPassConsumerThreads) {
+  if (XM == X_ATTN_FOLD) {
+    const int n_heads = st.ep.n_heads;
+    for (int e = tid; e < M * n_heads; e += kPassConsumerThreads) {
       const float* ml = pp.part_ml + (size_t)e * kAttnSplits * 2;  // e = m * n_heads + head
       float mj[kAttnSplits], lj[kAttnSplits];
       float mx = -INFINITY;
@@ -358,18 +368,18 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
     consumer_sync();
   }
 
-  // activation fragments of my next four units; kt_pref = k-tile of the next unit to prefetch
-  XRegs<CG> x0, x1, x2, x3;
+  // activation fragments of my next three units; kt_pref = k-tile of the next unit to prefetch
+  const XSource xs{st.X, st.gain, pp.part_o, st.ldx, st.ep.n_heads};
+  XRegs<CG> x0, x1, x2;
   int kt_pref = (kt_first + cls) % KT;
   auto prefetch = [&](XRegs<CG>& x, int i) {
-    load_xregs<CG, HD>(x, st, pp, sc, head0, n_heads_local, M, kt_pref, g, q, i < my_n);
+    load_xregs<CG, HD, XM>(x, xs, sc, M, kt_pref, g, q, i < my_n);
     kt_pref += kChunkUnits;
     if (kt_pref >= KT) kt_pref -= KT;
   };
   prefetch(x0, 0);
   prefetch(x1, 1);
   prefetch(x2, 2);
-  prefetch(x3, 3);
   if (st.rms_mode == RMS_FROM_PARTS && tid < M) {
     // the stage that produced the residual stream left one sum of squares per 128-feature group;
     // issued after the activation loads, read by the epilogue behind at least one barrier
@@ -378,7 +388,7 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
     sh->inv_rms[tid] = rsqrtf(s / (float)st.K + pp.eps);
   }
 
-  int i = 0;          // my next unit is number cls + 4 i
+  int i = 0;          // my next unit is number cls + kChunkUnits * i
   int seg_begin = 0;  // in units from ub64
   int grp = grp0;
   int seg_kt0 = kt_first;  // k-tile at seg_begin
@@ -390,19 +400,18 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
     const bool owner = starts_group && !whole;
 
     // the old residual values this thread will add to, fetched now so that they are there at the end
-    float2 hold[2 * CG];
+    float2 hold[CG];
 #pragma unroll
-    for (int j = 0; j < 2 * CG; ++j) hold[j] = make_float2(0.f, 0.f);
-    if (starts_group && st.ep.mode == EPI_RESID) {
+    for (int j = 0; j < CG; ++j) hold[j] = make_float2(0.f, 0.f);
+    if (starts_group && epi_mode == EPI_RESID) {
 #pragma unroll
-      for (int j = 0; j < 2 * CG; ++j) {
+      for (int j = 0; j < CG; ++j) {
         const int it = tid + j * kPassConsumerThreads;
         const int ch = it & 1, ln = (it >> 1) & 31, rc = it >> 6;
         const int cg = rc % CG, tile = rc / CG;
         const int m = cg * 8 + 2 * (ln & 3) + ch;
         const int rt = grp * kUnitTiles + tile;
-        hold[j] = make_float2(0.f, 0.f);
-        if (m < M && rt < st.NT) {
+        if (m < M && rt < NT) {
           const float* hp = st.ep.out + (size_t)m * st.ep.out_ld + 16 * rt + (ln >> 2);
           hold[j] = make_float2(ld_act(hp), ld_act(hp + 8));
         }
@@ -418,9 +427,8 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
         for (int e = 0; e < 4; ++e) acc[r][cg][e] = 0.f;
 
     bool warp_ok = true;
+    int kt = seg_kt0 + (cls + kChunkUnits * i - seg_begin);  // k-tile of my next unit while it lies in this segment
     while (warp_ok && i < my_n && cls + kChunkUnits * i < seg_end) {
-      const unsigned gc = chunk_base + (unsigned)i;
-      const unsigned slot = gc % (unsigned)n_slots, parity = (gc / (unsigned)n_slots) & 1u;
       // Lanes leave the polling loop at different times.  mma.sync needs the whole warp
       // converged, so the vote below is both the warp-uniform outcome and the reconvergence point.
       warp_ok = __all_sync(0xffffffffu, bounded_wait([&] { return mbar_try_wait(&sh->full[slot], parity); }, pp.sync,
@@ -430,11 +438,18 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
       uint4 a[4];
 #pragma unroll
       for (int r = 0; r < 4; ++r) a[r] = tiles[r * 32 + lane];
+      // the RMSNorm gain at this unit's columns (a constant vector: ordinary cached loads)
+      float2 g0 = make_float2(1.f, 1.f), g1 = make_float2(1.f, 1.f);
+      if (xs.gain != nullptr) {
+        const float* gp = xs.gain + kt * 16 + 2 * q;
+        g0 = __ldg(reinterpret_cast<const float2*>(gp));
+        g1 = __ldg(reinterpret_cast<const float2*>(gp + 8));
+      }
 #pragma unroll
       for (int cg = 0; cg < CG; ++cg) {
         uint32_t bh0, bl0, bh1, bl1;
-        split_pack(x0.lo8[cg].x * x0.g0.x, x0.lo8[cg].y * x0.g0.y, bh0, bl0);
-        split_pack(x0.hi8[cg].x * x0.g1.x, x0.hi8[cg].y * x0.g1.y, bh1, bl1);
+        split_pack(x0.lo8[cg].x * g0.x, x0.lo8[cg].y * g0.y, bh0, bl0);
+        split_pack(x0.hi8[cg].x * g1.x, x0.hi8[cg].y * g1.y, bh1, bl1);
 #pragma unroll
         for (int r = 0; r < 4; ++r) {
           mma_bf16_16816(acc[r][cg], a[r], bh0, bh1);
@@ -448,14 +463,18 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
       asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->empty[slot]);
+      if (++slot == (unsigned)n_slots) {
+        slot = 0;
+        parity ^= 1u;
+      }
       x0 = x1;
       x1 = x2;
-      x2 = x3;
-      prefetch(x3, i + 4);
+      prefetch(x2, i + 3);
       ++i;
+      kt += kChunkUnits;
     }
 
-    // ---- end of the segment: add the four class partials, then finish the group or post ----
+    // ---- end of the segment: add the class partials, then finish the group or post ----
 #pragma unroll
     for (int r = 0; r < 4; ++r)
 #pragma unroll
@@ -488,7 +507,7 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
       float2* my_post = reinterpret_cast<float2*>(pp.split_partials) + (size_t)cta * (kUnitTiles * CG * 64);
       const int n_parts = owner ? sh->n_parts : 0;
 #pragma unroll
-      for (int j = 0; j < 2 * CG; ++j) {
+      for (int j = 0; j < CG; ++j) {
         const int it = tid + j * kPassConsumerThreads;
         const int ch = it & 1;
         const int ln = (it >> 1) & 31;
@@ -496,8 +515,8 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
         const int cg = rc % CG, tile = rc / CG;
         float v0 = 0.f, v1 = 0.f;
 #pragma unroll
-        for (int c4 = 0; c4 < 4; ++c4) {
-          const float* p = reinterpret_cast<const float*>(red + ((c4 * kUnitTiles + tile) * CG + cg) * 32 + ln);
+        for (int c8 = 0; c8 < kClasses; ++c8) {
+          const float* p = reinterpret_cast<const float*>(red + ((c8 * kUnitTiles + tile) * CG + cg) * 32 + ln);
           v0 += p[ch];
           v1 += p[ch + 2];
         }
@@ -514,9 +533,9 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
         const int m = cg * 8 + 2 * (ln & 3) + ch;
         const int rt = grp * kUnitTiles + tile;
         float sq = 0.f;
-        if (m < M && rt < st.NT) {
+        if (m < M && rt < NT) {
           const float inv = sh->inv_rms[m];
-          if (st.ep.mode == EPI_RESID) {
+          if (epi_mode == EPI_RESID) {
             float* hp = st.ep.out + (size_t)m * st.ep.out_ld + 16 * rt + (ln >> 2);
             const float n0 = hold[j].x + v0 * inv, n1 = hold[j].y + v1 * inv;
             hp[0] = n0;
@@ -554,8 +573,6 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   // once the slot has been filled: an earlier arrival would be counted for the slot's previous
   // use and let the producer overwrite tiles another warp is still reading.
   if (my_n < n_chunks) {
-    const unsigned gc = chunk_base + (unsigned)(n_chunks - 1);
-    const unsigned slot = gc % (unsigned)n_slots, parity = (gc / (unsigned)n_slots) & 1u;
     if (bounded_wait([&] { return mbar_try_wait(&sh->full[slot], parity); }, pp.sync, &sh->abort, PASS_ERR_SLOT_FULL)) {
       __syncwarp();
       if (lane == 0) mbar_arrive(&sh->empty[slot]);
@@ -565,21 +582,23 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
 }
 
 // ---- attention stage --------------------------------------------------------------------------
-// One item = (head, split j, row group), handled by half a CTA.  Split j owns the 64-key chunks
-// j, j + kAttnSplits, ... of the head (chunk grid fixed in absolute key index) and walks them in
-// order with a running max and sum per row; it leaves an un-normalised partial (max, sum, o) per
-// row.  The O-projection that follows combines the kAttnSplits partials in split order while it
-// loads its activations, so nothing waits on another CTA inside this stage.  A row's numbers
-// depend only on its own position: rows that cannot see a chunk skip it entirely.
+// One item = (head, split j, row group), handled by half the consumer threads.  Split j owns the
+// 64-key chunks j, j + kAttnSplits, ... of the head (chunk grid fixed in absolute key index) and
+// walks them in order with a running max and sum per row; it leaves an un-normalised partial
+// (max, sum, o) per row.  The O-projection that follows combines the kAttnSplits partials in split
+// order while it loads its activations, so nothing waits on another CTA inside this stage.  A
+// row's numbers depend only on its own position: rows that cannot see a chunk skip it entirely.
+// Thread t of the half: scores as (key t/4, quarter t%4 of the head dimension), output as
+// (dimension t%HD, key half t/HD); the two key halves are added (first + second) at the end.
 template <int HD>
 __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassShared* sh, unsigned char* smem, int half,
                                int htid, int head, int split, int b) {
   using KT = __nv_bfloat16;
   constexpr int C = kAttnChunk;
-  KT* sV = reinterpret_cast<KT*>(smem);               // [C][HD]
+  static_assert(kHalfThreads == 4 * C, "one key per four threads");
+  KT* sV = reinterpret_cast<KT*>(smem);               // [C][HD]; at the end the second key half's o [R][HD] fp32
   float* sQ = reinterpret_cast<float*>(sV + C * HD);  // [R][HD]
   float* sS = sQ + kPassAttnR * HD;                   // [R][C]
-  int* s_pos = sh->attn_pos[half];
   float* s_m = sh->attn_m[half];
   float* s_l = sh->attn_l[half];
   float* s_a = sh->attn_a[half];
@@ -587,28 +606,31 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
   const int row0 = b * R;
   const int n_heads = st.ep.n_heads;
   const size_t d_model = (size_t)n_heads * HD;
+  auto pos_of = [&](int i) { return (row0 + i < pp.M) ? sh->row_pos[row0 + i] : -1; };
 
+  int max_pos = -1;
+  for (int i = 0; i < R; ++i) max_pos = max(max_pos, pos_of(i));
+  const int seq = sh->row_seq[row0];
   if (htid < R) {
-    s_pos[htid] = (row0 + htid < pp.M) ? ld_act(pp.row_pos + row0 + htid) : -1;
     s_m[htid] = -INFINITY;
     s_l[htid] = 0.f;
   }
-  half_sync(half);
-  int max_pos = -1;
-  for (int i = 0; i < R; ++i) max_pos = max(max_pos, s_pos[i]);
-  const int seq = ld_act(pp.row_seq + row0);
-  for (int e = htid; e < R * HD; e += 128) {
+  for (int e = htid; e < R * HD; e += kHalfThreads) {
     const int i = e / HD, d = e - i * HD;
-    sQ[e] = (s_pos[i] >= 0) ? ld_act(st.X + (size_t)(row0 + i) * d_model + head * HD + d) : 0.f;
+    sQ[e] = (pos_of(i) >= 0) ? ld_act(st.X + (size_t)(row0 + i) * d_model + head * HD + d) : 0.f;
   }
 
-  float o[kPassAttnR];  // thread d < HD: o[i][d]
+  constexpr int QD = HD / 4;    // dimensions of a key one thread multiplies
+  constexpr int KV4 = QD / 8;   // uint4 of bf16 per thread
+  constexpr int VPR = HD / 8;   // uint4 per V row
+  const int key = htid >> 2, qr = htid & 3;
+  const int od = htid % HD, okh = htid / HD;        // output dimension and key half (HD = 128: 0/1; HD = 64: 0..3 -> use 2)
+  constexpr int KH = (kHalfThreads / HD) >= 2 ? 2 : 1;  // key halves in the output phase
+  const bool o_active = okh < KH;
+  float o[kPassAttnR];
 #pragma unroll
   for (int i = 0; i < kPassAttnR; ++i) o[i] = 0.f;
 
-  constexpr int KV4 = HD / 16;  // uint4 per half key row
-  constexpr int VPR = HD / 8;
-  const int key = htid >> 1, hf = htid & 1;
   for (int c = split; c * C <= max_pos; c += kAttnSplits) {
     const int key0 = c * C;
     const int nk_all = min(C, max_pos + 1 - key0);
@@ -619,18 +641,17 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
 #pragma unroll
     for (int j = 0; j < KV4; ++j) kreg[j] = make_uint4(0u, 0u, 0u, 0u);
     if (key < nk_all) {
-      const uint4* kp = reinterpret_cast<const uint4*>(gK + (size_t)key * HD + hf * (HD / 2));
+      const uint4* kp = reinterpret_cast<const uint4*>(gK + (size_t)key * HD + qr * QD);
 #pragma unroll
       for (int j = 0; j < KV4; ++j) kreg[j] = __ldcg(kp + j);
     }
-    half_sync(half);  // the previous chunk's sV and sS are no longer read (and sQ is complete)
-    for (int v = htid; v < nk_all * VPR; v += 128)
-      reinterpret_cast<uint4*>(sV)[v] = __ldcg(reinterpret_cast<const uint4*>(gV) + v);
+    half_sync(half);  // the previous chunk's sV and sS are no longer read, sQ and the row state are written
+    for (int v = htid; v < nk_all * VPR; v += kHalfThreads) cp_async16(reinterpret_cast<uint4*>(sV) + v, reinterpret_cast<const uint4*>(gV) + v);
     {
       float acc[kPassAttnR];
 #pragma unroll
       for (int i = 0; i < kPassAttnR; ++i) acc[i] = 0.f;
-      const float* qh = sQ + hf * (HD / 2);
+      const float* qh = sQ + qr * QD;
 #pragma unroll
       for (int j = 0; j < KV4; ++j) {
         const uint32_t w[4] = {kreg[j].x, kreg[j].y, kreg[j].z, kreg[j].w};
@@ -651,16 +672,18 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
 #pragma unroll
       for (int i = 0; i < kPassAttnR; ++i) {
         if (i < R) {
-          const float other = __shfl_xor_sync(0xffffffffu, acc[i], 1);
-          if (hf == 0) sS[i * C + key] = (acc[i] + other) * pp.attn_scale;
+          float s = acc[i];
+          s += __shfl_xor_sync(0xffffffffu, s, 1);  // quarters (0+1), (2+3)
+          s += __shfl_xor_sync(0xffffffffu, s, 2);  // then the two pairs
+          if (qr == 0) sS[i * C + key] = s * pp.attn_scale;
         }
       }
     }
     half_sync(half);
     {
-      const int w4 = htid >> 5, lane = htid & 31;
-      for (int i = w4; i < R; i += 4) {
-        const int nk = min(C, s_pos[i] + 1 - key0);
+      const int w8 = htid >> 5, lane = htid & 31;
+      for (int i = w8; i < R; i += kHalfThreads / 32) {
+        const int nk = min(C, pos_of(i) + 1 - key0);
         if (nk <= 0) {  // the row cannot see this chunk: leave its state alone
           if (lane == 0) s_a[i] = 1.f;
           sS[i * C + lane] = 0.f;
@@ -684,25 +707,38 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
         }
       }
     }
+    cp_async_wait_all();
     half_sync(half);
-    if (htid < HD) {
+    if (o_active) {
 #pragma unroll
       for (int i = 0; i < kPassAttnR; ++i)
         if (i < R) o[i] *= s_a[i];
-      for (int k2 = 0; k2 < nk_all; ++k2) {
-        const float v = __bfloat162float(sV[k2 * HD + htid]);
+      const int k_lo = okh * (C / KH), k_hi = min(nk_all, k_lo + C / KH);
+      for (int k2 = k_lo; k2 < k_hi; ++k2) {
+        const float v = __bfloat162float(sV[k2 * HD + od]);
 #pragma unroll
         for (int i = 0; i < kPassAttnR; ++i)
           if (i < R) o[i] = fmaf(sS[i * C + k2], v, o[i]);
       }
     }
   }
-  // the partial of every row of the group, also of rows that saw nothing here (sum 0)
-  if (htid < HD) {
+  // add the two key halves (first + second) and leave the partial of every row of the group,
+  // also of rows that saw nothing here (sum 0)
+  half_sync(half);
+  float* sO = reinterpret_cast<float*>(sV);
+  if (KH == 2 && o_active && okh == 1) {
 #pragma unroll
     for (int i = 0; i < kPassAttnR; ++i)
-      if (i < R && row0 + i < pp.M)
-        pp.part_o[((((size_t)(row0 + i)) * n_heads + head) * kAttnSplits + split) * HD + htid] = o[i];
+      if (i < R) sO[i * HD + od] = o[i];
+  }
+  half_sync(half);
+  if (o_active && okh == 0) {
+#pragma unroll
+    for (int i = 0; i < kPassAttnR; ++i)
+      if (i < R && row0 + i < pp.M) {
+        const float v = (KH == 2) ? o[i] + sO[i * HD + od] : o[i];
+        pp.part_o[((((size_t)(row0 + i)) * n_heads + head) * kAttnSplits + split) * HD + od] = v;
+      }
   }
   if (htid < R && row0 + htid < pp.M) {
     float* ml = pp.part_ml + ((((size_t)(row0 + htid)) * n_heads + head) * kAttnSplits + split) * 2;
@@ -717,19 +753,19 @@ __host__ __device__ constexpr size_t pass_attn_smem_half() {
   return (size_t)kAttnChunk * HD * 2 + (size_t)kPassAttnR * HD * 4 + (size_t)kPassAttnR * kAttnChunk * 4;
 }
 
-template <int HD>
+template <int CG, int HD>
 __host__ __device__ constexpr size_t pass_work_bytes() {
-  return (size_t)(kWorkScOff + kWorkScBytes) > 2 * pass_attn_smem_half<HD>() ? (size_t)(kWorkScOff + kWorkScBytes)
-                                                                              : 2 * pass_attn_smem_half<HD>();
+  return (size_t)(work_sc_off<CG>() + kWorkScBytes) > 2 * pass_attn_smem_half<HD>() ? (size_t)(work_sc_off<CG>() + kWorkScBytes)
+                                                                                    : 2 * pass_attn_smem_half<HD>();
 }
 
-// Dynamic shared memory: [ring: n_slots * 16 KB][work area][PassShared]
+// Dynamic shared memory: [ring: n_slots * 32 KB][work area][PassShared]
 template <int CG, int HD>
 __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, int n_slots) {
   extern __shared__ __align__(1024) unsigned char smem[];
   unsigned char* ring = smem;
   unsigned char* work = smem + (size_t)n_slots * kSlotBytes;
-  PassShared* sh = reinterpret_cast<PassShared*>(work + pass_work_bytes<HD>());
+  PassShared* sh = reinterpret_cast<PassShared*>(work + pass_work_bytes<CG, HD>());
   const int tid = threadIdx.x;
 
   if (tid == 0) {
@@ -740,12 +776,16 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
     sh->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  if (tid < kPassMaxRows) {  // where the rows sit does not change during the pass
+    sh->row_pos[tid] = tid < pp.M ? pp.row_pos[tid] : -1;
+    sh->row_seq[tid] = tid < pp.M ? pp.row_seq[tid] : 0;
+  }
   __syncthreads();
 
   if (tid >= kPassConsumerThreads) {
     // ================= producer warp: stream this CTA's share of every weight matrix =================
     if (tid == kPassConsumerThreads) {
-      unsigned gc = 0;
+      unsigned slot = 0, parity = 1u, issued = 0;
       bool ok = true;
       for (int s = 0; s < pp.n_stages && ok; ++s) {
         const StageDesc& st = pp.prog[s];
@@ -755,7 +795,6 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
         const unsigned char* src = reinterpret_cast<const unsigned char*>(st.W) + (size_t)ub * kUnitBytes;
         long long left = ue - ub;
         while (left > 0) {
-          const unsigned slot = gc % (unsigned)n_slots, parity = ((gc / (unsigned)n_slots) & 1u) ^ 1u;
           ok = bounded_wait([&] { return mbar_try_wait(&sh->empty[slot], parity); }, pp.sync, &sh->abort, PASS_ERR_SLOT_EMPTY);
           if (!ok) break;
           const unsigned n = left < kChunkUnits ? (unsigned)left : (unsigned)kChunkUnits;
@@ -763,16 +802,20 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
           bulk_load(ring + (size_t)slot * kSlotBytes, src, n * kUnitBytes, &sh->full[slot]);
           src += (size_t)n * kUnitBytes;
           left -= n;
-          ++gc;
+          ++issued;
+          if (++slot == (unsigned)n_slots) {
+            slot = 0;
+            parity ^= 1u;
+          }
         }
       }
       // nothing may still be landing in shared memory when the CTA exits: wait (bounded) for the
       // copies of the last n_slots slots that were issued
-      const unsigned first = gc > (unsigned)n_slots ? gc - (unsigned)n_slots : 0u;
-      for (unsigned j = first; j < gc; ++j) {
-        const unsigned slot = j % (unsigned)n_slots, parity = (j / (unsigned)n_slots) & 1u;
+      const unsigned first = issued > (unsigned)n_slots ? issued - (unsigned)n_slots : 0u;
+      for (unsigned j = first; j < issued; ++j) {
+        const unsigned sl = j % (unsigned)n_slots, par = (j / (unsigned)n_slots) & 1u;
         const unsigned long long t0 = global_ns();
-        while (!mbar_try_wait(&sh->full[slot], parity))
+        while (!mbar_try_wait(&sh->full[sl], par))
           if (global_ns() - t0 > kWaitLimitNs) break;
       }
     }
@@ -794,9 +837,12 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
     }
     if (sh->st.kind == ST_LINEAR) {
       // serial number of the stage over all launches: the posts of split groups carry it
-      linear_stage<CG, HD>(pp, sh, ring, n_slots, work, chunk_base, bar_base + (unsigned)s + 1u);
+      if (sh->st.x_mode == X_PLAIN)
+        linear_stage<CG, HD, X_PLAIN>(pp, sh, ring, n_slots, work, chunk_base, bar_base + (unsigned)s + 1u);
+      else
+        linear_stage<CG, HD, X_ATTN_FOLD>(pp, sh, ring, n_slots, work, chunk_base, bar_base + (unsigned)s + 1u);
     } else {
-      const int half = tid >> 7, htid = tid & 127;
+      const int half = tid / kHalfThreads, htid = tid % kHalfThreads;
       const int n_heads = sh->st.ep.n_heads;
       const int n_groups = (pp.M + pp.rows_per_seq - 1) / pp.rows_per_seq;
       const int items = kAttnSplits * n_heads * n_groups;
