@@ -358,6 +358,7 @@ cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool w
   pp.row_seq = c->plan.row_seq;
   pp.eps = c->cfg.rms_eps;
   pp.attn_scale = 1.0f / std::sqrt((float)c->cfg.head_dim);
+  pp.zero = 0u;
   pp.part_o = c->part_o;
   pp.part_ml = c->part_ml;
   pp.split_partials = c->split_partials;

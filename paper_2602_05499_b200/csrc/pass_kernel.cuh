@@ -91,6 +91,7 @@ struct PassParams {
   const int* row_seq;
   float eps;
   float attn_scale;
+  unsigned zero;  // always 0: lets code build values the compiler cannot fold away
   // scratch
   float* part_o;          // attention partials [rows][head][kAttnSplits][head_dim], not normalised
   float* part_ml;         // [rows][head][kAttnSplits][2] running max and sum
@@ -107,6 +108,15 @@ __device__ __forceinline__ void mbar_init(uint64_t* bar, unsigned count) {
 }
 __device__ __forceinline__ void mbar_arrive(uint64_t* bar) {
   asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.shared::cta.b64 st, [%0];\n}" ::"r"(smem_u32(bar)) : "memory");
+}
+// Arrival without ordering semantics of its own, at an address that depends on `dep`.  A
+// releasing arrival would first wait for every earlier memory operation of the thread, including
+// activation loads still on their way from L2, and the consumer loop then runs at one L2 round
+// trip per unit.  The only accesses that must be over before a slot is handed back are the
+// shared-memory reads of its tiles: the caller passes a value computed from the registers those
+// reads filled (and masked to zero), so the arrival cannot issue before they have returned.
+__device__ __forceinline__ void mbar_arrive_relaxed_after(uint64_t* bar, unsigned dep) {
+  asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.relaxed.cta.shared::cta.b64 st, [%0];\n}" ::"r"(smem_u32(bar) + dep) : "memory");
 }
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t* bar, unsigned bytes) {
   asm volatile("{\n .reg .b64 st;\n mbarrier.arrive.expect_tx.shared::cta.b64 st, [%0], %1;\n}" ::"r"(smem_u32(bar)), "r"(bytes)
@@ -232,6 +242,7 @@ __device__ __forceinline__ void unit_range(long long n_units, int cta, int n_cta
 template <int CG>
 struct XRegs {
   float2 lo8[CG], hi8[CG];  // x[m][16kt + 2q .. +1] and x[m][16kt + 2q + 8 .. +9], m = 8 cg + g
+  float2 g0, g1;            // the RMSNorm gain at the same columns (1 when the stage has no norm)
 };
 
 struct XSource {  // the fields of the stage an activation load needs, kept in registers
@@ -247,6 +258,13 @@ struct XSource {  // the fields of the stage an activation load needs, kept in r
 template <int CG, int HD, int XM>
 __device__ __forceinline__ void load_xregs(XRegs<CG>& x, const XSource& xs, const float* sc, int M, int kt, int g, int q,
                                            bool valid) {
+  x.g0 = make_float2(1.f, 1.f);
+  x.g1 = make_float2(1.f, 1.f);
+  if (valid && xs.gain != nullptr) {  // asked for together with the activations: a first touch misses L1
+    const float* gp = xs.gain + kt * 16 + 2 * q;
+    x.g0 = __ldg(reinterpret_cast<const float2*>(gp));
+    x.g1 = __ldg(reinterpret_cast<const float2*>(gp + 8));
+  }
 #pragma unroll
   for (int cg = 0; cg < CG; ++cg) {
     const int m = cg * 8 + g;
@@ -380,12 +398,26 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   prefetch(x0, 0);
   prefetch(x1, 1);
   prefetch(x2, 2);
-  if (st.rms_mode == RMS_FROM_PARTS && tid < M) {
-    // the stage that produced the residual stream left one sum of squares per 128-feature group;
-    // issued after the activation loads, read by the epilogue behind at least one barrier
-    float s = 0.f;
-    for (int gi = 0; gi < st.ssq_groups; ++gi) s += ld_act(pp.ssq_part + gi * kPassMaxRows + tid);
-    sh->inv_rms[tid] = rsqrtf(s / (float)st.K + pp.eps);
+  if (st.rms_mode == RMS_FROM_PARTS && warp == kPassConsumerWarps - 1) {
+    // The stage that produced the residual stream left one sum of squares per 128-feature group.
+    // One warp adds them: every lane asks for all its terms at once (a serial chain of loads
+    // would hold this warp, and with it the ring, for dozens of L2 round trips); per lane the
+    // terms are added in group order, across lanes with the fixed xor tree.
+    float part[kPassMaxRows];
+#pragma unroll
+    for (int m = 0; m < kPassMaxRows; ++m) part[m] = 0.f;
+    for (int gi = lane; gi < st.ssq_groups; gi += 32) {
+#pragma unroll
+      for (int m = 0; m < kPassMaxRows; ++m)
+        if (m < M) part[m] += ld_act(pp.ssq_part + gi * kPassMaxRows + m);
+    }
+#pragma unroll
+    for (int m = 0; m < kPassMaxRows; ++m) {
+      if (m < M) {
+        const float s = warp_sum(part[m]);
+        if (lane == 0) sh->inv_rms[m] = rsqrtf(s / (float)st.K + pp.eps);
+      }
+    }
   }
 
   int i = 0;          // my next unit is number cls + kChunkUnits * i
@@ -438,13 +470,7 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
       uint4 a[4];
 #pragma unroll
       for (int r = 0; r < 4; ++r) a[r] = tiles[r * 32 + lane];
-      // the RMSNorm gain at this unit's columns (a constant vector: ordinary cached loads)
-      float2 g0 = make_float2(1.f, 1.f), g1 = make_float2(1.f, 1.f);
-      if (xs.gain != nullptr) {
-        const float* gp = xs.gain + kt * 16 + 2 * q;
-        g0 = __ldg(reinterpret_cast<const float2*>(gp));
-        g1 = __ldg(reinterpret_cast<const float2*>(gp + 8));
-      }
+      const float2 g0 = x0.g0, g1 = x0.g1;
 #pragma unroll
       for (int cg = 0; cg < CG; ++cg) {
         uint32_t bh0, bl0, bh1, bl1;
@@ -456,13 +482,16 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
           mma_bf16_16816(acc[r][cg], a[r], bl0, bl1);
         }
       }
-      // The tiles were read through the generic proxy; the slot is about to be handed back to
-      // the producer, whose next bulk copy writes it through the async proxy.  Without this
-      // fence the arrival could take effect while the reads were still pending, and a refill
-      // then replaced 64-byte pieces of a tile under them (seen as rare wrong rows at full speed).
-      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&sh->empty[slot]);
+      // Hand the slot back once the tile reads above have returned: the producer's next bulk
+      // copy overwrites it through the async proxy, and an arrival that overtook pending reads
+      // let a refill replace 64-byte pieces of a tile under them (rare wrong rows at full speed).
+      {
+        unsigned dep = a[0].x ^ a[1].y ^ a[2].z ^ a[3].w;
+        asm volatile("" : "+r"(dep)::"memory");
+        dep &= pp.zero;  // zero at run time, unknown to the compiler
+        __syncwarp();
+        if (lane == 0) mbar_arrive_relaxed_after(&sh->empty[slot], dep);
+      }
       if (++slot == (unsigned)n_slots) {
         slot = 0;
         parity ^= 1u;
