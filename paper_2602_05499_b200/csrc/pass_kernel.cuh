@@ -619,7 +619,8 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
 // row's numbers depend only on its own position: rows that cannot see a chunk skip it entirely.
 // Thread t of the half: scores as (key t/4, quarter t%4 of the head dimension), output as
 // (dimension t%HD, key half t/HD); the two key halves are added (first + second) at the end.
-template <int HD>
+// RM = compile-time row capacity (the per-row registers are arrays of RM entries).
+template <int HD, int RM>
 __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassShared* sh, unsigned char* smem, int half,
                                int htid, int head, int split, int b) {
   using KT = __nv_bfloat16;
@@ -644,10 +645,16 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
     s_m[htid] = -INFINITY;
     s_l[htid] = 0.f;
   }
-  for (int e = htid; e < R * HD; e += kHalfThreads) {
-    const int i = e / HD, d = e - i * HD;
-    sQ[e] = (pos_of(i) >= 0) ? ld_act(st.X + (size_t)(row0 + i) * d_model + head * HD + d) : 0.f;
-  }
+  // q rows of this head, 16 bytes at a time, straight into shared memory (rows that carry nothing: zeros)
+  auto fetch_q = [&]() {
+    for (int e = htid; e < R * (HD / 4); e += kHalfThreads) {
+      const int i = e / (HD / 4), d4 = e - i * (HD / 4);
+      if (pos_of(i) >= 0)
+        cp_async16(sQ + i * HD + d4 * 4, st.X + (size_t)(row0 + i) * d_model + head * HD + d4 * 4);
+      else
+        *reinterpret_cast<float4*>(sQ + i * HD + d4 * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+    }
+  };
 
   constexpr int QD = HD / 4;    // dimensions of a key one thread multiplies
   constexpr int KV4 = QD / 8;   // uint4 of bf16 per thread
@@ -656,9 +663,9 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
   const int od = htid % HD, okh = htid / HD;        // output dimension and key half (HD = 128: 0/1; HD = 64: 0..3 -> use 2)
   constexpr int KH = (kHalfThreads / HD) >= 2 ? 2 : 1;  // key halves in the output phase
   const bool o_active = okh < KH;
-  float o[kPassAttnR];
+  float o[RM];
 #pragma unroll
-  for (int i = 0; i < kPassAttnR; ++i) o[i] = 0.f;
+  for (int i = 0; i < RM; ++i) o[i] = 0.f;
 
   for (int c = split; c * C <= max_pos; c += kAttnSplits) {
     const int key0 = c * C;
@@ -674,12 +681,17 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
 #pragma unroll
       for (int j = 0; j < KV4; ++j) kreg[j] = __ldcg(kp + j);
     }
-    half_sync(half);  // the previous chunk's sV and sS are no longer read, sQ and the row state are written
+    half_sync(half);  // the previous chunk's sV and sS are no longer read, the row state is written
+    if (c == split) fetch_q();  // first chunk: all three requests (K, q, V) are in flight together
     for (int v = htid; v < nk_all * VPR; v += kHalfThreads) cp_async16(reinterpret_cast<uint4*>(sV) + v, reinterpret_cast<const uint4*>(gV) + v);
+    if (c == split) {
+      cp_async_wait_all();  // q (and V) have landed; make q visible to the whole half
+      half_sync(half);
+    }
     {
-      float acc[kPassAttnR];
+      float acc[RM];
 #pragma unroll
-      for (int i = 0; i < kPassAttnR; ++i) acc[i] = 0.f;
+      for (int i = 0; i < RM; ++i) acc[i] = 0.f;
       const float* qh = sQ + qr * QD;
 #pragma unroll
       for (int j = 0; j < KV4; ++j) {
@@ -689,7 +701,7 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
           const float k0 = __uint_as_float(w[e] << 16), k1 = __uint_as_float(w[e] & 0xffff0000u);
           const int d = j * 8 + e * 2;
 #pragma unroll
-          for (int i = 0; i < kPassAttnR; ++i) {
+          for (int i = 0; i < RM; ++i) {
             if (i < R) {
               const float2 qv = *reinterpret_cast<const float2*>(qh + i * HD + d);
               acc[i] = fmaf(k0, qv.x, acc[i]);
@@ -699,7 +711,7 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
         }
       }
 #pragma unroll
-      for (int i = 0; i < kPassAttnR; ++i) {
+      for (int i = 0; i < RM; ++i) {
         if (i < R) {
           float s = acc[i];
           s += __shfl_xor_sync(0xffffffffu, s, 1);  // quarters (0+1), (2+3)
@@ -740,13 +752,13 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
     half_sync(half);
     if (o_active) {
 #pragma unroll
-      for (int i = 0; i < kPassAttnR; ++i)
+      for (int i = 0; i < RM; ++i)
         if (i < R) o[i] *= s_a[i];
       const int k_lo = okh * (C / KH), k_hi = min(nk_all, k_lo + C / KH);
       for (int k2 = k_lo; k2 < k_hi; ++k2) {
         const float v = __bfloat162float(sV[k2 * HD + od]);
 #pragma unroll
-        for (int i = 0; i < kPassAttnR; ++i)
+        for (int i = 0; i < RM; ++i)
           if (i < R) o[i] = fmaf(sS[i * C + k2], v, o[i]);
       }
     }
@@ -757,13 +769,13 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
   float* sO = reinterpret_cast<float*>(sV);
   if (KH == 2 && o_active && okh == 1) {
 #pragma unroll
-    for (int i = 0; i < kPassAttnR; ++i)
+    for (int i = 0; i < RM; ++i)
       if (i < R) sO[i * HD + od] = o[i];
   }
   half_sync(half);
   if (o_active && okh == 0) {
 #pragma unroll
-    for (int i = 0; i < kPassAttnR; ++i)
+    for (int i = 0; i < RM; ++i)
       if (i < R && row0 + i < pp.M) {
         const float v = (KH == 2) ? o[i] + sO[i * HD + od] : o[i];
         pp.part_o[((((size_t)(row0 + i)) * n_heads + head) * kAttnSplits + split) * HD + od] = v;
@@ -879,7 +891,13 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
       for (int it = blockIdx.x * 2 + half; it < items; it += gridDim.x * 2) {
         const int split = it % kAttnSplits;
         const int hb = it / kAttnSplits;
-        attention_item<HD>(sh->st, pp, sh, my, half, htid, hb % n_heads, split, hb / n_heads);
+        const int hd_ = hb % n_heads, b_ = hb / n_heads;
+        if (pp.rows_per_seq <= 2)
+          attention_item<HD, 2>(sh->st, pp, sh, my, half, htid, hd_, split, b_);
+        else if (pp.rows_per_seq <= 8)
+          attention_item<HD, 8>(sh->st, pp, sh, my, half, htid, hd_, split, b_);
+        else
+          attention_item<HD, 16>(sh->st, pp, sh, my, half, htid, hd_, split, b_);
       }
     }
     ok = consumers_agree_ok(sh);
