@@ -41,6 +41,9 @@ WORKLOADS = {
     "c1-tiny-greedy-k4": (si.TINY, 2, 4, 16, 64),
     "7b-4layers-greedy-k4": (si.LLAMA7B_4L, 2, 4, 64, 64),
 }
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
+# capture summarised under profiles/ (null until a capture of the current kernel exists)
+TRAFFIC = {}
 PAPER_CONTEXT = "paper reports 1.32x-1.5x over vanilla decoding for LLaMA-2-13B/70B on unstated hardware"
 
 
@@ -260,16 +263,31 @@ def main():
     ar_pass_gbs = (ar_t["weight_bytes"] + ar_t["kv_bytes"]) / (ar_t["decode_ms"] * 1e-3) / 1e9
     assert ar.tokens == out.tokens, "speculative greedy output differs from autoregressive output"
 
-    # ---- dominant kernel, live (CUDA events inside the library around back-to-back launches) --
+    # ---- dominant kernel, live: the whole-pass kernel (one launch = one forward pass), timed with a
+    # CUDA-event pair around every launch on the library's stream; the draft pass is the launch the
+    # decode phase spends most of its time in (k draft passes per verify pass)
     peak, peak_src = measured_peak_gbs()
-    names = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
     per_kernel = {}
-    for rows in (1, 2, k + 1):
-        for which, nm in enumerate(names):
-            ms, nbytes = eng.sdfp_time_linear(which, rows, 64 if which < 4 else 16)
-            per_kernel[f"{nm}@M={rows}"] = {"us": round(ms * 1e3, 2), "GB/s": round(nbytes / ms / 1e6, 1)}
-    gu_ms, gu_bytes = eng.sdfp_time_linear(2, k + 1, 128)
-    kernel_gbs = gu_bytes / gu_ms / 1e6
+    mid = plen + n_new // 2                      # a context in the middle of the generation
+    uses_pass = shape.dtype == "bf16" and not (args.flags & (pkg.FLAG_NO_PASS_KERNEL | pkg.FLAG_FMA_GEMM))
+    if uses_pass:
+        for name, draft, rows in (("draft_pass@M=1", True, 1), ("draft_pass@M=2", True, 2),
+                                  ("verify_pass@M=%d" % (k + 1), False, k + 1), ("ar_pass@M=1", False, 1)):
+            ms, nbytes = eng.sdfp_time_pass(draft, rows, mid, 24)
+            per_kernel[name] = {"us": round(ms * 1e3, 1), "GB/s": round(nbytes / ms / 1e6, 1),
+                                "bytes": int(nbytes), "frac_of_peak": round(nbytes / ms / 1e6 / peak, 3)}
+        dom_ms, dom_bytes = eng.sdfp_time_pass(True, 1, mid, 48)
+        dom_name = "pass_kernel (draft pass: %d of %d layers + lm-head, M=1, context %d)" % (
+            shape.n_layers - len(skip), shape.n_layers, mid)
+    else:
+        names = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
+        for rows in (1, k + 1):
+            for which, nm in enumerate(names):
+                ms, nbytes = eng.sdfp_time_linear(which, rows, 64 if which < 4 else 16)
+                per_kernel[f"{nm}@M={rows}"] = {"us": round(ms * 1e3, 2), "GB/s": round(nbytes / ms / 1e6, 1)}
+        dom_ms, dom_bytes = eng.sdfp_time_linear(2, k + 1, 128)
+        dom_name = "linear kernel (gate/up, M=%d)" % (k + 1)
+    kernel_gbs = dom_bytes / dom_ms / 1e6
 
     # ---- reduce over ranks --------------------------------------------------------------------------
     vals = torch.tensor([dec_ms, step_ms, wall_s], device=dev, dtype=torch.float64)
@@ -312,9 +330,10 @@ def main():
                     "note": "whole sdfp_generate call: prompt copy, prefill of both caches, decode, token copy"},
             "gpu_launches": int(launches_all),
             "clocks": clocks,
-            "roofline": {"bound": "hbm", "kernel": "linear_mma_kernel (gate/up, M=%d)" % (k + 1),
+            "roofline": {"bound": "hbm", "kernel": dom_name,
                          "achieved": kernel_gbs, "peak": peak, "unit": "GB/s", "frac": kernel_gbs / peak,
-                         "peak_source": peak_src, "traffic": None,
+                         "peak_source": peak_src, "traffic": TRAFFIC.get(args.workload) if uses_pass else None,
+                         "algorithmic_bytes_per_launch": int(dom_bytes), "us_per_launch": dom_ms * 1e3,
                          "pass_level": {"spec_GB/s": spec_pass_gbs, "spec_frac_of_peak": spec_pass_gbs / peak,
                                         "spec_frac_of_8TB/s": spec_pass_gbs / 8000.0,
                                         "ar_GB/s": ar_pass_gbs, "ar_frac_of_peak": ar_pass_gbs / peak,

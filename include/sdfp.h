@@ -211,6 +211,20 @@ int sdfp_get_timing(const sdfp_ctx *ctx, sdfp_timing *out);
 int sdfp_time_linear(sdfp_ctx *ctx, int32_t which, int32_t rows, int32_t iters,
                      float *ms_per_launch, int64_t *weight_bytes_per_launch);
 
+/*
+ * Micro-benchmark hook for the roofline report of the whole-pass kernel (bf16 models without
+ * SDFP_FLAG_NO_PASS_KERNEL; SDFP_ESTATE otherwise).  Runs `iters` forward passes of `rows`
+ * rows (1..16) of sequence slot 0 at positions position.. through the target (draft == 0) or
+ * the draft model, lm-head included, and returns the average duration of ONE launch of the
+ * pass kernel in milliseconds (a CUDA-event pair around every launch, on the context's stream)
+ * together with the bytes such a launch has to move: the weights of the layers it runs and of
+ * the lm-head, the K/V of those layers for positions 0..position+rows-1, and the K/V rows it
+ * writes.  The token ids fed are 0; the K/V cache of slot 0 is overwritten from `position` on
+ * (in Section II-A's terms: a timing-only verification pass whose result is discarded).
+ */
+int sdfp_time_pass(sdfp_ctx *ctx, int32_t draft, int32_t rows, int32_t position, int32_t iters,
+                   float *ms_per_launch, int64_t *bytes_per_launch);
+
 const char *sdfp_last_error(const sdfp_ctx *ctx);
 void sdfp_destroy(sdfp_ctx *ctx);
 

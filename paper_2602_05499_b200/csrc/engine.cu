@@ -1021,6 +1021,57 @@ extern "C" int sdfp_get_timing(const sdfp_ctx* c, sdfp_timing* out) {
   return 0;
 }
 
+extern "C" int sdfp_time_pass(sdfp_ctx* c, int32_t draft, int32_t rows, int32_t position, int32_t iters,
+                              float* ms_per_launch, int64_t* bytes_per_launch) {
+  if (!c) return SDFP_EINVAL;
+  const sdfp_config& g = c->cfg;
+  if (!ms_per_launch || !bytes_per_launch) return fail(c, SDFP_EINVAL, "sdfp_time_pass: NULL pointer");
+  if (!c->use_pass) return fail(c, SDFP_ESTATE, "sdfp_time_pass: this context does not use the whole-pass kernel");
+  if (rows < 1 || rows > kPassMaxRows || iters < 1 || iters > 256 || position < 0 || position + rows > g.max_seq)
+    return fail(c, SDFP_EINVAL, "sdfp_time_pass: bad argument");
+  CU_OK(c, cudaMemsetAsync(c->fwd_tok, 0, (size_t)kMaxRows * 4, c->stream));
+  PassDesc pd{};
+  pd.kind = PASS_TOKENS;
+  pd.seq = 0;
+  pd.start = position;
+  pd.count = rows;
+  pd.src = c->fwd_tok;
+  std::vector<cudaEvent_t> ev(2 * (size_t)iters, nullptr);
+  for (auto& e : ev) CU_OK(c, cudaEventCreate(&e));
+  auto plan = [&]() -> cudaError_t {
+    return launch(c, plan_embed_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs,
+                  (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
+                  reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, g.d_model);
+  };
+  cudaError_t err = cudaSuccess;
+  for (int i = 0; i < 3 && err == cudaSuccess; ++i) {  // warm-up
+    err = plan();
+    if (err == cudaSuccess) err = run_pass(c, draft != 0, rows, rows, true);
+  }
+  for (int i = 0; i < iters && err == cudaSuccess; ++i) {
+    err = plan();  // fresh residual rows every time, outside the timed interval
+    if (err == cudaSuccess) err = cudaEventRecord(ev[2 * i], c->stream);
+    if (err == cudaSuccess) err = run_pass(c, draft != 0, rows, rows, true);
+    if (err == cudaSuccess) err = cudaEventRecord(ev[2 * i + 1], c->stream);
+  }
+  if (err == cudaSuccess) err = cudaStreamSynchronize(c->stream);
+  double total = 0.0;
+  for (int i = 0; i < iters && err == cudaSuccess; ++i) {
+    float ms = 0.f;
+    err = cudaEventElapsedTime(&ms, ev[2 * i], ev[2 * i + 1]);
+    total += ms;
+  }
+  for (auto& e : ev) cudaEventDestroy(e);
+  CU_OK(c, err);
+  if (int r = check_pass_error(c)) return r;
+  *ms_per_launch = (float)(total / iters);
+  const int64_t layers = draft ? kept_layers(c) : g.n_layers;
+  const int64_t kv_tok = 2LL * g.d_model * (int64_t)c->esz;
+  *bytes_per_launch = layers * layer_weight_bytes(c) + lm_head_bytes(c) + layers * kv_tok * ((int64_t)position + rows) +
+                      layers * kv_tok * rows;
+  return 0;
+}
+
 extern "C" int sdfp_time_linear(sdfp_ctx* c, int32_t which, int32_t rows, int32_t iters, float* ms_per_launch,
                                 int64_t* weight_bytes_per_launch) {
   if (!c) return SDFP_EINVAL;
