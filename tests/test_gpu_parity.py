@@ -299,6 +299,44 @@ def test_per_operation_kernels_agree_with_pass_kernel(shape, draw):
     check_stream_against_oracle(m, prompt[0].tolist(), g2.tokens[0])
 
 
+def test_pass_kernel_long_context_blocks(l7b4):
+    """Whole-pass kernel at a context of several 64-key chunks: 16-row passes (two column groups,
+    one attention item walking several chunks) give bit for bit what single-row passes give, and
+    both match the oracle."""
+    eng, m = l7b4
+    toks = si.make_prompts(m.vocab, 1, 208, seed=16)[0].tolist()
+    one = np.concatenate([eng.sdfp_forward_logits(toks[i:i + 1], i) for i in range(208)])
+    blk = np.concatenate([eng.sdfp_forward_logits(toks[s:s + 16], s) for s in range(0, 208, 16)])
+    assert np.array_equal(one.view(np.uint32), blk.view(np.uint32))
+    five = np.concatenate([eng.sdfp_forward_logits(toks[s:s + 5], s) for s in range(100, 200, 5)])
+    assert np.array_equal(one[100:200].view(np.uint32), five.view(np.uint32))
+    ref = orc.CachedLM(m, max_seq=256).feed(toks, 0).numpy()
+    assert max(rel_l2(blk[r], ref[r]) for r in range(208)) < 1e-2
+
+
+@pytest.mark.parametrize("k", [8])
+def test_greedy_wide_verify_equals_ar(tiny_bf16, l7b4, k):
+    """k = 8: the verify pass carries 9 rows (two column groups) while the autoregressive pass
+    carries one; the streams must still be identical."""
+    for eng, m in (tiny_bf16, l7b4):
+        prompt = si.make_prompts(m.vocab, 1, 70, seed=17)
+        out = eng.sdfp_generate(prompt, k, 40)
+        ar = eng.sdfp_generate(prompt, 0, 40)
+        assert out.tokens[0] == ar.tokens[0]
+        check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+
+
+def test_time_pass_hook(l7b4):
+    eng, m = l7b4
+    ms, nbytes = eng.sdfp_time_pass(False, 5, 100, 4)
+    d, f, v, L = 4096, 11008, 32000, 4
+    want = L * (4 * d * d + 3 * d * f) * 2 + v * d * 2 + L * 2 * d * 2 * (100 + 5) + L * 2 * d * 2 * 5
+    assert nbytes == want and 0.05 < ms < 50
+    ms_d, nbytes_d = eng.sdfp_time_pass(True, 1, 100, 4)          # the draft keeps layers 0 and 3
+    assert nbytes_d == 2 * (4 * d * d + 3 * d * f) * 2 + v * d * 2 + 2 * 2 * d * 2 * 101 + 2 * 2 * d * 2
+    assert ms_d < ms
+
+
 def test_fma_and_tensor_paths_agree_closely():
     """The CUDA-core comparison path and the tensor-core path compute the same model."""
     shape = si.LLAMA7B_4L
