@@ -140,6 +140,20 @@ def oracle_sample(shape, w_cpu, skip, k, prompt_len_sample, new_tokens, n_thread
     return len(res.tokens) / (t2 - t1), t2 - t1, t1 - t0, res
 
 
+def reduce_over_ranks(times, counts, device, world):
+    """Replicas share nothing but this: times are reduced with MAX over ranks (the job is as slow as
+    its slowest replica), counts with SUM (whole-job totals).  Works on any backend (nccl on the
+    GPUs, gloo in the CPU test)."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(times), device=device, dtype=torch.float64)
+    c = torch.tensor(list(counts), device=device, dtype=torch.float64)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+        dist.all_reduce(c, op=dist.ReduceOp.SUM)
+    return [float(x) for x in t.tolist()], [float(x) for x in c.tolist()]
+
+
 def run_reference(args, workload):
     """--impl reference: the oracle on the host cores (rank 0 only)."""
     import torch
@@ -292,13 +306,8 @@ def main():
     kernel_gbs = dom_bytes / dom_ms / 1e6
 
     # ---- reduce over ranks --------------------------------------------------------------------------
-    vals = torch.tensor([dec_ms, step_ms, wall_s], device=dev, dtype=torch.float64)
-    tok = torch.tensor([float(tokens), float(launches)], device=dev, dtype=torch.float64)
-    if world > 1:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-        dist.all_reduce(tok, op=dist.ReduceOp.SUM)
-    dec_ms_max, step_ms_max, wall_max = [float(x) for x in vals.tolist()]
-    tokens_all, launches_all = [float(x) for x in tok.tolist()]
+    (dec_ms_max, step_ms_max, wall_max), (tokens_all, launches_all) = reduce_over_ranks(
+        [dec_ms, step_ms, wall_s], [float(tokens), float(launches)], dev, world)
     value = tokens_all / (dec_ms_max * 1e-3)
     e2e_value = tokens_all / wall_max
     spec_pass_gbs = (wbytes + kvbytes) / (dec_ms * 1e-3) / 1e9

@@ -54,6 +54,9 @@ LLAMA13B = ModelShape("llama2-13b-shape-bf16", 40, 5120, 40, 128, 13824, 32000, 
 # LLAMA7B, small enough for the CPU oracle to finish in seconds.
 LLAMA7B_4L = replace(LLAMA7B, name="llama2-7b-shape-4layers-bf16", n_layers=4)
 
+# The 13B shape cut to two layers: d = 5120 (40 heads), FFN 13824, for shape coverage of the kernels.
+LLAMA13B_2L = replace(LLAMA13B, name="llama2-13b-shape-2layers-bf16", n_layers=2)
+
 MASTER_SEED = 20260205
 PROMPT_SEED = 1234
 

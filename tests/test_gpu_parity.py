@@ -337,6 +337,43 @@ def test_time_pass_hook(l7b4):
     assert ms_d < ms
 
 
+def test_13b_shape_layers():
+    """d = 5120, 40 heads x 128, FFN 13824: the 13B configuration's linear and attention shapes
+    (two layers deep so that the oracle finishes in seconds), logits and greedy streams."""
+    shape = si.LLAMA13B_2L
+    eng, m, _ = make_pair(shape, (0,), max_seq=256, k_max=8, draw_device="cuda:0")
+    try:
+        toks = si.make_prompts(shape.vocab, 1, 150, seed=18)[0].tolist()
+        got, ref = _logits_both(eng, m, toks, [64, 33, 1, 5, 16, 31])
+        assert max(rel_l2(got[r], ref[r]) for r in range(150)) < 1e-2
+        prompt = si.make_prompts(shape.vocab, 1, 130, seed=19)
+        out = eng.sdfp_generate(prompt, 4, 32)
+        ar = eng.sdfp_generate(prompt, 0, 32)
+        assert out.tokens[0] == ar.tokens[0]
+        check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+    finally:
+        eng.close()
+
+
+def test_batch_rows_are_independent_bf16():
+    """Three sequences with k = 4 are 15 rows: they run in the whole-pass kernel as three row
+    groups.  A sequence's tokens and acceptance counts must not depend on the others."""
+    eng, m, _ = make_pair(si.TINY_BF16, (1, 2), max_batch=3, k_max=4)
+    try:
+        prompts = si.make_prompts(m.vocab, 3, 24, seed=41)
+        out = eng.sdfp_generate(prompts, 4, 40)
+        ar = eng.sdfp_generate(prompts, 0, 40)
+        assert out.tokens == ar.tokens
+        for b in range(3):
+            solo = eng.sdfp_generate(prompts[b:b + 1], 4, 40)
+            assert solo.tokens[0] == out.tokens[b]
+            acc_b = [int(a) for a, d in zip(out.stats[:, b, 1], out.stats[:, b, 0]) if d > 0]
+            assert acc_b == solo.stats[:, 0, 1].tolist()
+            check_stream_against_oracle(m, prompts[b].tolist(), out.tokens[b])
+    finally:
+        eng.close()
+
+
 def test_fma_and_tensor_paths_agree_closely():
     """The CUDA-core comparison path and the tensor-core path compute the same model."""
     shape = si.LLAMA7B_4L
