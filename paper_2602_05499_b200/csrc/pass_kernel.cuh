@@ -647,18 +647,22 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
     s_m[htid] = -INFINITY;
     s_l[htid] = 0.f;
   }
-  // q rows of this head, 16 bytes at a time, straight into shared memory (rows that carry nothing: zeros)
+  // q rows of this head, 16 bytes at a time, straight into shared memory (rows that carry nothing:
+  // zeros).  Inside quarter r of a row (QD dimensions) the dimensions are rotated by 8 r: the four
+  // threads that work on one key read the same offset of the four quarters at once, and the
+  // rotation puts those four addresses into different banks.
+  constexpr int QD = HD / 4;  // dimensions of a key one thread multiplies
   auto fetch_q = [&]() {
     for (int e = htid; e < R * (HD / 4); e += kHalfThreads) {
       const int i = e / (HD / 4), d4 = e - i * (HD / 4);
+      const int d = d4 * 4, r = d / QD, phys = r * QD + (d - r * QD + 8 * r) % QD;
       if (pos_of(i) >= 0)
-        cp_async16(sQ + i * HD + d4 * 4, st.X + (size_t)(row0 + i) * d_model + head * HD + d4 * 4);
+        cp_async16(sQ + i * HD + phys, st.X + (size_t)(row0 + i) * d_model + head * HD + d);
       else
-        *reinterpret_cast<float4*>(sQ + i * HD + d4 * 4) = make_float4(0.f, 0.f, 0.f, 0.f);
+        *reinterpret_cast<float4*>(sQ + i * HD + phys) = make_float4(0.f, 0.f, 0.f, 0.f);
     }
   };
 
-  constexpr int QD = HD / 4;    // dimensions of a key one thread multiplies
   constexpr int KV4 = QD / 8;   // uint4 of bf16 per thread
   constexpr int VPR = HD / 8;   // uint4 per V row
   const int key = htid >> 2, qr = htid & 3;
@@ -694,18 +698,17 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
       float acc[RM];
 #pragma unroll
       for (int i = 0; i < RM; ++i) acc[i] = 0.f;
-      const float* qh = sQ + qr * QD;
 #pragma unroll
       for (int j = 0; j < KV4; ++j) {
         const uint32_t w[4] = {kreg[j].x, kreg[j].y, kreg[j].z, kreg[j].w};
 #pragma unroll
         for (int e = 0; e < 4; ++e) {
           const float k0 = __uint_as_float(w[e] << 16), k1 = __uint_as_float(w[e] & 0xffff0000u);
-          const int d = j * 8 + e * 2;
+          const int d = qr * QD + (j * 8 + e * 2 + 8 * qr) % QD;  // where fetch_q put this dimension
 #pragma unroll
           for (int i = 0; i < RM; ++i) {
             if (i < R) {
-              const float2 qv = *reinterpret_cast<const float2*>(qh + i * HD + d);
+              const float2 qv = *reinterpret_cast<const float2*>(sQ + i * HD + d);
               acc[i] = fmaf(k0, qv.x, acc[i]);
               acc[i] = fmaf(k1, qv.y, acc[i]);
             }
