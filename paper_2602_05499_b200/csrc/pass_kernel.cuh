@@ -7,10 +7,11 @@
 // 16 rows), and a 7B layer is four weight sweeps of 5..28 us each.  As separate launches every
 // sweep pays a ramp-up and a tail; here the weight stream never stops:
 //   * One producer warp per CTA walks the whole stage list and copies this CTA's share of every
-//     weight matrix into a ring of 16 KB shared-memory slots with bulk asynchronous copies
+//     weight matrix into a ring of 32 KB shared-memory slots with bulk asynchronous copies
 //     (cp.async.bulk + mbarrier transaction counts).  Weights do not depend on activations, so the
 //     producer runs ahead of the consumers across stage boundaries, through the grid barriers,
-//     as far as the ring allows (160 KB per SM, ~24 MB over the GPU).
+//     as far as the ring allows (three slots, 96 KB per SM, ~14 MB over the GPU; two slots when a
+//     pass carries more than 8 rows and the work area is larger).
 //   * Sixteen consumer warps take the slots in order, feed the tiles to mma.sync.m16n8k16 (weights
 //     are the A operand, tokens the 8-wide B operand) and run the fused epilogues.
 //   * Stages are separated by a grid barrier (arrival counter in global memory, bounded spin).
@@ -702,15 +703,18 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
       for (int j = 0; j < KV4; ++j) {
         const uint32_t w[4] = {kreg[j].x, kreg[j].y, kreg[j].z, kreg[j].w};
 #pragma unroll
-        for (int e = 0; e < 4; ++e) {
+        for (int e = 0; e < 4; e += 2) {
           const float k0 = __uint_as_float(w[e] << 16), k1 = __uint_as_float(w[e] & 0xffff0000u);
-          const int d = qr * QD + (j * 8 + e * 2 + 8 * qr) % QD;  // where fetch_q put this dimension
+          const float k2 = __uint_as_float(w[e + 1] << 16), k3 = __uint_as_float(w[e + 1] & 0xffff0000u);
+          const int d = qr * QD + (j * 8 + e * 2 + 8 * qr) % QD;  // where fetch_q put these four dimensions
 #pragma unroll
           for (int i = 0; i < RM; ++i) {
             if (i < R) {
-              const float2 qv = *reinterpret_cast<const float2*>(sQ + i * HD + d);
+              const float4 qv = *reinterpret_cast<const float4*>(sQ + i * HD + d);
               acc[i] = fmaf(k0, qv.x, acc[i]);
               acc[i] = fmaf(k1, qv.y, acc[i]);
+              acc[i] = fmaf(k2, qv.z, acc[i]);
+              acc[i] = fmaf(k3, qv.w, acc[i]);
             }
           }
         }
@@ -760,7 +764,21 @@ __device__ void attention_item(const StageDesc& st, const PassParams& pp, PassSh
       for (int i = 0; i < RM; ++i)
         if (i < R) o[i] *= s_a[i];
       const int k_lo = okh * (C / KH), k_hi = min(nk_all, k_lo + C / KH);
-      for (int k2 = k_lo; k2 < k_hi; ++k2) {
+      int k2 = k_lo;
+      for (; k2 + 4 <= k_hi; k2 += 4) {  // four keys per step, added in key order
+        const float v0 = __bfloat162float(sV[(k2 + 0) * HD + od]), v1 = __bfloat162float(sV[(k2 + 1) * HD + od]);
+        const float v2 = __bfloat162float(sV[(k2 + 2) * HD + od]), v3 = __bfloat162float(sV[(k2 + 3) * HD + od]);
+#pragma unroll
+        for (int i = 0; i < RM; ++i)
+          if (i < R) {
+            const float4 p4 = *reinterpret_cast<const float4*>(sS + i * C + k2);
+            o[i] = fmaf(p4.x, v0, o[i]);
+            o[i] = fmaf(p4.y, v1, o[i]);
+            o[i] = fmaf(p4.z, v2, o[i]);
+            o[i] = fmaf(p4.w, v3, o[i]);
+          }
+      }
+      for (; k2 < k_hi; ++k2) {
         const float v = __bfloat162float(sV[k2 * HD + od]);
 #pragma unroll
         for (int i = 0; i < RM; ++i)
