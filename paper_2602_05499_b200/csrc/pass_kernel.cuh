@@ -74,13 +74,11 @@ struct StageDesc {
 // what a wait that gave up leaves in PassSync::error
 enum PassError { PASS_OK = 0, PASS_ERR_GRID_BARRIER = 1, PASS_ERR_SLOT_FULL = 2, PASS_ERR_SLOT_EMPTY = 3, PASS_ERR_SPLIT_FLAG = 4 };
 
-struct PassSync {      // one per context, in global memory, zero-initialised
-  unsigned bar_count;  // grid-barrier arrivals, ever increasing (wraps): serial * grid when barrier `serial` is complete
-  unsigned pad0[31];
-  unsigned bar_gen;    // serial number of the last barrier that completed; written by its last arriver
-  unsigned pad1[31];
+struct PassSync {                // one per context, in global memory, zero-initialised
+  unsigned long long bar_count;  // grid-barrier arrivals of all launches so far: serial * grid when barrier `serial` is complete
+  unsigned pad0[30];
   int error;           // first PassError seen, sticky
-  unsigned pad2[31];
+  unsigned pad1[31];
 };
 
 struct PassParams {
@@ -93,6 +91,7 @@ struct PassParams {
   float eps;
   float attn_scale;
   unsigned zero;  // always 0: lets code build values the compiler cannot fold away
+  int pf_chunks;  // how many chunks ahead of the ring the producer prefetches weights into L2
   // scratch
   float* part_o;          // attention partials [rows][head][kAttnSplits][head_dim], not normalised
   float* part_ml;         // [rows][head][kAttnSplits][2] running max and sum
@@ -132,12 +131,23 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t* bar, unsigned parity) {
       : "memory");
   return ok != 0;
 }
-// Bulk asynchronous copy global -> shared, completion counted in bytes on an mbarrier.
-// Both addresses and the size are multiples of 16 bytes.
-__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar) {
-  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];" ::"r"(smem_u32(dst)),
-               "l"(src), "r"(bytes), "r"(smem_u32(bar))
+__device__ __forceinline__ uint64_t l2_policy_evict_first() {
+  uint64_t pol;
+  asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(pol));
+  return pol;
+}
+// Bulk asynchronous copy global -> shared, completion counted in bytes on an mbarrier; `pol` says
+// how long L2 should keep the lines.  Both addresses and the size are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_load(void* dst, const void* src, unsigned bytes, uint64_t* bar, uint64_t pol) {
+  asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1], %2, [%3], %4;" ::"r"(
+                   smem_u32(dst)),
+               "l"(src), "r"(bytes), "r"(smem_u32(bar)), "l"(pol)
                : "memory");
+}
+// Ask for a range of global memory to be brought into L2 (nothing waits for it).  Address and size
+// are multiples of 16 bytes.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* src, unsigned bytes) {
+  asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(src), "r"(bytes) : "memory");
 }
 // 16-byte asynchronous copy global -> shared through L2 only (attention's V tiles)
 __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
@@ -152,10 +162,13 @@ __device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
 __device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
   asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
 }
-__device__ __forceinline__ unsigned atom_add_release(unsigned* p, unsigned v) {
-  unsigned old;
-  asm volatile("atom.add.release.gpu.global.u32 %0, [%1], %2;" : "=r"(old) : "l"(p), "r"(v) : "memory");
-  return old;
+__device__ __forceinline__ unsigned long long ld_relaxed(const unsigned long long* p) {
+  unsigned long long v;
+  asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];" : "=l"(v) : "l"(p) : "memory");
+  return v;
+}
+__device__ __forceinline__ void red_add_relaxed(unsigned long long* p, unsigned long long v) {
+  asm volatile("red.relaxed.gpu.global.add.u64 [%0], %1;" ::"l"(p), "l"(v) : "memory");
 }
 __device__ __forceinline__ unsigned long long global_ns() {
   unsigned long long t;
@@ -175,6 +188,7 @@ struct PassShared {
   StageDesc st_next;  // the next one, fetched while the running stage works
   float inv_rms[kPassMaxRows];
   int row_pos[kPassMaxRows], row_seq[kPassMaxRows];  // fixed for the whole pass
+  unsigned long long bar_base;
   int abort;     // set by whichever thread gives up a wait
   int decision;  // abort as sampled by thread 0 between two consumer barriers: uniform for all
   float attn_m[2][kPassAttnR], attn_l[2][kPassAttnR], attn_a[2][kPassAttnR];
@@ -216,21 +230,21 @@ __device__ __forceinline__ bool bounded_wait(Pred pred, PassSync* sync, volatile
 }
 
 // ---- grid barrier (consumer threads of every CTA) ------------------------------------------------
-// Everything the consumer threads of this CTA wrote before is visible to every CTA after.  The
-// arrivals go to one counter; the CTA that completes the count publishes the barrier's serial
-// number in a word of its own cache line, which is all the others poll, so polling never collides
-// with arrivals.  (Measured against an all-gather of per-CTA words polled by 148 threads per CTA:
-// this one is 1.7% faster per pass.)  Counter and serial numbers only grow (wrap-safe comparison).
-__device__ __forceinline__ bool grid_barrier(PassSync* sync, unsigned serial, PassShared* sh) {
+// Everything the consumer threads of this CTA wrote before is visible to every CTA after.  One
+// 64-bit counter in global memory only ever grows: barrier number `serial` (counted over all
+// launches of the context) is complete when it reads serial * grid.  A CTA arrives with
+// a reduction that returns nothing and then polls the counter with relaxed loads; the fences
+// before the arrival and after the last poll carry the ordering.  The critical path after the last
+// arrival is one trip of the reduction to L2 and one poll, where a scheme in which the last
+// arriver publishes a flag adds the return of its atomic, another fence and a store.
+__device__ __forceinline__ bool grid_barrier(PassSync* sync, unsigned long long serial, PassShared* sh) {
   consumer_sync();
   if (threadIdx.x == 0) {
+    const unsigned long long target = serial * gridDim.x;
     __threadfence();
-    const unsigned old = atom_add_release(&sync->bar_count, 1u);
-    if (old + 1u == serial * gridDim.x) {
-      st_release(&sync->bar_gen, serial);
-    } else {
-      bounded_wait([&] { return (int)(ld_acquire(&sync->bar_gen) - serial) >= 0; }, sync, &sh->abort, PASS_ERR_GRID_BARRIER);
-    }
+    red_add_relaxed(&sync->bar_count, 1ull);
+    bounded_wait([&] { return ld_relaxed(&sync->bar_count) >= target; }, sync, &sh->abort, PASS_ERR_GRID_BARRIER);
+    __threadfence();
     sh->decision = sh->abort;
   }
   consumer_sync();
@@ -840,6 +854,10 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
     sh->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
+  // Barriers completed by earlier launches: the counter is a multiple of the grid size when a
+  // launch starts and stays below the next multiple until every CTA, this one included, has
+  // arrived at the launch's first barrier.
+  if (tid == 32) sh->bar_base = ld_relaxed(&pp.sync->bar_count) / gridDim.x;
   if (tid < kPassMaxRows) {  // where the rows sit does not change during the pass
     sh->row_pos[tid] = tid < pp.M ? pp.row_pos[tid] : -1;
     sh->row_seq[tid] = tid < pp.M ? pp.row_seq[tid] : 0;
@@ -849,28 +867,57 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
   if (tid >= kPassConsumerThreads) {
     // ================= producer warp: stream this CTA's share of every weight matrix =================
     if (tid == kPassConsumerThreads) {
-      unsigned slot = 0, parity = 1u, issued = 0;
+      // Two cursors walk the same list of chunks (a chunk = up to kChunkUnits units of one stage):
+      // `ld` copies a chunk into the ring as soon as a slot is free, `pf` runs up to pf_chunks
+      // chunks further ahead and only asks for them to be brought into L2.  The ring holds about
+      // 2 us of weight traffic, a stage boundary (partial posts, epilogue, grid barrier, the next
+      // stage's activations) costs the consumers several times that; with the prefetch the memory
+      // keeps streaming through those gaps and the ring refills from L2 afterwards.  The copies
+      // into the ring mark their lines evict-first, so what L2 keeps is what has not been used yet.
+      struct Cursor {
+        int s;
+        const unsigned char* src;
+        long long left;
+      };
+      auto advance = [&](Cursor& c) {  // to the next linear stage that has units for this CTA
+        while (c.left == 0 && c.s < pp.n_stages) {
+          if (++c.s == pp.n_stages) break;
+          const StageDesc& st = pp.prog[c.s];
+          if (st.kind != ST_LINEAR) continue;
+          long long ub, ue;
+          unit_range((long long)st.n_groups * st.KT, blockIdx.x, gridDim.x, ub, ue);
+          c.src = reinterpret_cast<const unsigned char*>(st.W) + (size_t)ub * kUnitBytes;
+          c.left = ue - ub;
+        }
+      };
+      const uint64_t pol_first = l2_policy_evict_first();  // a weight is read once per pass
+      Cursor ld{-1, nullptr, 0}, pf{-1, nullptr, 0};
+      advance(ld);
+      advance(pf);
+      unsigned slot = 0, parity = 1u, issued = 0, ahead = 0;
       bool ok = true;
-      for (int s = 0; s < pp.n_stages && ok; ++s) {
-        const StageDesc& st = pp.prog[s];
-        if (st.kind != ST_LINEAR) continue;
-        long long ub, ue;
-        unit_range((long long)st.n_groups * st.KT, blockIdx.x, gridDim.x, ub, ue);
-        const unsigned char* src = reinterpret_cast<const unsigned char*>(st.W) + (size_t)ub * kUnitBytes;
-        long long left = ue - ub;
-        while (left > 0) {
-          ok = bounded_wait([&] { return mbar_try_wait(&sh->empty[slot], parity); }, pp.sync, &sh->abort, PASS_ERR_SLOT_EMPTY);
-          if (!ok) break;
-          const unsigned n = left < kChunkUnits ? (unsigned)left : (unsigned)kChunkUnits;
-          mbar_arrive_expect_tx(&sh->full[slot], n * kUnitBytes);
-          bulk_load(ring + (size_t)slot * kSlotBytes, src, n * kUnitBytes, &sh->full[slot]);
-          src += (size_t)n * kUnitBytes;
-          left -= n;
-          ++issued;
-          if (++slot == (unsigned)n_slots) {
-            slot = 0;
-            parity ^= 1u;
-          }
+      while (ld.s < pp.n_stages) {
+        while (ahead < (unsigned)pp.pf_chunks && pf.s < pp.n_stages) {
+          const unsigned n = pf.left < kChunkUnits ? (unsigned)pf.left : (unsigned)kChunkUnits;
+          if (ahead >= (unsigned)n_slots) bulk_prefetch_l2(pf.src, n * kUnitBytes);  // nearer chunks are copied at once anyway
+          pf.src += (size_t)n * kUnitBytes;
+          pf.left -= n;
+          advance(pf);
+          ++ahead;
+        }
+        ok = bounded_wait([&] { return mbar_try_wait(&sh->empty[slot], parity); }, pp.sync, &sh->abort, PASS_ERR_SLOT_EMPTY);
+        if (!ok) break;
+        const unsigned n = ld.left < kChunkUnits ? (unsigned)ld.left : (unsigned)kChunkUnits;
+        mbar_arrive_expect_tx(&sh->full[slot], n * kUnitBytes);
+        bulk_load(ring + (size_t)slot * kSlotBytes, ld.src, n * kUnitBytes, &sh->full[slot], pol_first);
+        ld.src += (size_t)n * kUnitBytes;
+        ld.left -= n;
+        advance(ld);
+        ++issued;
+        if (ahead > 0) --ahead;
+        if (++slot == (unsigned)n_slots) {
+          slot = 0;
+          parity ^= 1u;
         }
       }
       // nothing may still be landing in shared memory when the CTA exits: wait (bounded) for the
@@ -887,9 +934,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
   }
 
   // ================= consumer warps =================
-  // Serial number of the last barrier of the previous launch; nothing changes it before every
-  // CTA of this launch has arrived at the first barrier, i.e. has read it here.
-  const unsigned bar_base = *reinterpret_cast<volatile unsigned*>(&pp.sync->bar_gen);
+  const unsigned long long bar_base = sh->bar_base;
   unsigned chunk_base = 0;
   bool ok = true;
   constexpr int kDescWords = (int)(sizeof(StageDesc) / sizeof(int));
@@ -914,9 +959,9 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
       // launch's first stage): only a launch's last stage and the next launch's first would
       // otherwise collide.
       if (sh->st.x_mode == X_PLAIN)
-        linear_stage<CG, HD, X_PLAIN>(pp, sh, ring, n_slots, work, chunk_base, 2u * (bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u);
+        linear_stage<CG, HD, X_PLAIN>(pp, sh, ring, n_slots, work, chunk_base, 2u * ((unsigned)bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u);
       else
-        linear_stage<CG, HD, X_ATTN_FOLD>(pp, sh, ring, n_slots, work, chunk_base, 2u * (bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u);
+        linear_stage<CG, HD, X_ATTN_FOLD>(pp, sh, ring, n_slots, work, chunk_base, 2u * ((unsigned)bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u);
     } else {
       const int half = tid / kHalfThreads, htid = tid % kHalfThreads;
       const int n_heads = sh->st.ep.n_heads;
@@ -936,8 +981,8 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
       }
     }
     if (desc_w >= 0 && desc_w < kDescWords) reinterpret_cast<int*>(&sh->st_next)[desc_w] = next_word;
-    ok = consumers_agree_ok(sh);
-    if (ok && s + 1 < pp.n_stages) ok = grid_barrier(pp.sync, bar_base + (unsigned)(s + 1), sh);
+    // the barrier also tells every thread whether a wait of this CTA gave up (the CTA still arrives)
+    ok = (s + 1 < pp.n_stages) ? grid_barrier(pp.sync, bar_base + (unsigned long long)(s + 1), sh) : consumers_agree_ok(sh);
   }
 }
 
