@@ -95,8 +95,7 @@ struct sdfp_ctx {
   StageDesc *prog_t = nullptr, *prog_d = nullptr;  // device: stage lists of the target and of the draft
   int n_prog_t = 0, n_prog_d = 0;
   PassSync* psync = nullptr;
-  float* split_partials = nullptr;
-  unsigned* split_flags = nullptr;
+  ulonglong2* split_partials = nullptr;
   float* ssq_part = nullptr;
   int pass_slots[3] = {0, 0, 0};  // ring slots of the instantiation with 1 and with 2 column groups
   size_t pass_smem = 0;
@@ -379,7 +378,6 @@ cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool w
   pp.part_o = c->part_o;
   pp.part_ml = c->part_ml;
   pp.split_partials = c->split_partials;
-  pp.split_flags = c->split_flags;
   pp.ssq_part = c->ssq_part;
   pp.sync = c->psync;
   const bool hd128 = c->cfg.head_dim == 128;
@@ -694,8 +692,7 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
     return bail(r);
   if (c->use_pass) {
     if ((r = dev_alloc(c, &c->psync, 1, true)) ||
-        (r = dev_alloc(c, &c->split_partials, (size_t)c->pass_grid * kUnitTiles * 2 * 64 * 2, true)) ||
-        (r = dev_alloc(c, &c->split_flags, (size_t)c->pass_grid, true)) ||
+        (r = dev_alloc(c, &c->split_partials, (size_t)c->pass_grid * kUnitTiles * 2 * 64, true)) ||
         (r = dev_alloc(c, &c->ssq_part, (size_t)kSsqMaxGroups * kPassMaxRows, true)) || (r = build_programs(c)))
       return bail(r);
   }
@@ -746,7 +743,7 @@ int check_pass_error(sdfp_ctx* c) {
   CU_OK(c, cudaStreamSynchronize(c->stream));
   if (ps.error == 0) return 0;
   cudaMemsetAsync(c->psync, 0, sizeof(PassSync), c->stream);
-  cudaMemsetAsync(c->split_flags, 0, (size_t)c->pass_grid * sizeof(unsigned), c->stream);
+  cudaMemsetAsync(c->split_partials, 0, (size_t)c->pass_grid * kUnitTiles * 2 * 64 * sizeof(ulonglong2), c->stream);
   cudaStreamSynchronize(c->stream);
   static const char* const what[] = {"", "grid barrier", "weight slot never filled", "weight slot never freed",
                                      "partial sum of a split group never posted"};

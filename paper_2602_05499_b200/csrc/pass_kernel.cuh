@@ -24,7 +24,10 @@
 // shares differ by at most one unit (4 KB).  A range cuts groups at arbitrary k: a group that
 // spans several CTAs is finished by the CTA that holds its beginning (which reaches it last),
 // after the others have posted their partial sums to global scratch; partials are added in CTA
-// order, so the result does not depend on timing.
+// order, so the result does not depend on timing.  A post is written as 64-bit words that hold a
+// value and the stage's serial number side by side: the owner sees a value as soon as its word
+// has arrived and no fence or flag stands between the poster's stores and the owner's loads (a
+// fence issued under the weight stream takes 1-5 us).
 //
 // Inside a CTA the 16 consumer warps are 8 k-classes x 2 tile halves: the unit with index
 // (range start + c + 8i) belongs to class c, and warp (c, t) multiplies its tiles 4t..4t+3.  The
@@ -95,8 +98,7 @@ struct PassParams {
   // scratch
   float* part_o;          // attention partials [rows][head][kAttnSplits][head_dim], not normalised
   float* part_ml;         // [rows][head][kAttnSplits][2] running max and sum
-  float* split_partials;  // [grid][kUnitTiles * CG * 64 * 2]
-  unsigned* split_flags;  // [grid]
+  ulonglong2* split_partials;  // [grid][kUnitTiles * CG * 64] packets of two (value, stage serial) words
   float* ssq_part;        // [kSsqMaxGroups][kPassMaxRows]
   PassSync* sync;
 };
@@ -154,13 +156,20 @@ __device__ __forceinline__ void cp_async16(void* dst, const void* src) {
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(smem_u32(dst)), "l"(src) : "memory");
 }
 __device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_all;" ::: "memory"); }
-__device__ __forceinline__ unsigned ld_acquire(const unsigned* p) {
-  unsigned v;
-  asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+// (value, serial) packets of the split-group posts: a 64-bit word is written and read whole, so a
+// reader that finds the stage's serial number in a word has the value that came with it
+__device__ __forceinline__ void st_packet(ulonglong2* p, float v0, float v1, unsigned serial) {
+  const unsigned long long hi = (unsigned long long)serial << 32;
+  asm volatile("st.relaxed.gpu.global.v2.u64 [%0], {%1, %2};" ::"l"(p), "l"(hi | __float_as_uint(v0)), "l"(hi | __float_as_uint(v1))
+               : "memory");
+}
+__device__ __forceinline__ ulonglong2 ld_packet(const ulonglong2* p) {
+  ulonglong2 v;
+  asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(v.x), "=l"(v.y) : "l"(p) : "memory");
   return v;
 }
-__device__ __forceinline__ void st_release(unsigned* p, unsigned v) {
-  asm volatile("st.release.gpu.global.u32 [%0], %1;" ::"l"(p), "r"(v) : "memory");
+__device__ __forceinline__ bool packet_is(const ulonglong2& v, unsigned serial) {
+  return (unsigned)(v.x >> 32) == serial && (unsigned)(v.y >> 32) == serial;
 }
 __device__ __forceinline__ unsigned long long ld_relaxed(const unsigned long long* p) {
   unsigned long long v;
@@ -227,6 +236,21 @@ __device__ __forceinline__ bool bounded_wait(Pred pred, PassSync* sync, volatile
       }
     }
   }
+}
+
+// Wait for one packet of a post, polls a little apart.  Out of line: the common case (the packet
+// is there at the first look) should not pay registers for this loop.
+__device__ __noinline__ ulonglong2 wait_packet(const ulonglong2* src, unsigned serial, PassSync* sync, volatile int* s_abort) {
+  ulonglong2 pk = make_ulonglong2(0ull, 0ull);
+  bounded_wait(
+      [&] {
+        pk = ld_packet(src);
+        if (packet_is(pk, serial)) return true;
+        __nanosleep(50);
+        return false;
+      },
+      sync, s_abort, PASS_ERR_SPLIT_FLAG);
+  return pk;
 }
 
 // ---- grid barrier (consumer threads of every CTA) ------------------------------------------------
@@ -540,7 +564,9 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
         if (c2 < n_cta) unit_range(n_units, c2, n_cta, b2, e2);
         const bool beyond = (c2 >= n_cta) || (b2 >= grp_end);
         const bool part = !beyond && e2 > b2;  // an empty range posts nothing
-        if (part) bounded_wait([&] { return ld_acquire(pp.split_flags + c2) == epoch; }, pp.sync, &sh->abort, PASS_ERR_SPLIT_FLAG);
+        // one lane per posting CTA waits for the packet that CTA's last thread writes; the others
+        // are then there too or about to be, and every reader checks its own packets anyway
+        if (part) wait_packet(pp.split_partials + (size_t)c2 * (kUnitTiles * CG * 64) + (kPassConsumerThreads * CG - 1), epoch, pp.sync, &sh->abort);
         const unsigned mask = __ballot_sync(0xffffffffu, part);
         if (part) sh->parts[n + __popc(mask & ((1u << lane) - 1u))] = c2;
         n += __popc(mask);
@@ -551,7 +577,7 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
     if (!consumers_agree_ok(sh)) return;
 
     {
-      float2* my_post = reinterpret_cast<float2*>(pp.split_partials) + (size_t)cta * (kUnitTiles * CG * 64);
+      ulonglong2* my_post = pp.split_partials + (size_t)cta * (kUnitTiles * CG * 64);
       const int n_parts = owner ? sh->n_parts : 0;
 #pragma unroll
       for (int j = 0; j < CG; ++j) {
@@ -568,14 +594,15 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
           v1 += p[ch + 2];
         }
         if (!starts_group) {
-          my_post[it] = make_float2(v0, v1);
+          st_packet(my_post + it, v0, v1, epoch);
           continue;
         }
         for (int k2 = 0; k2 < n_parts; ++k2) {
-          const float2 o =
-              __ldcg(reinterpret_cast<const float2*>(pp.split_partials) + (size_t)sh->parts[k2] * (kUnitTiles * CG * 64) + it);
-          v0 += o.x;
-          v1 += o.y;
+          const ulonglong2* src = pp.split_partials + (size_t)sh->parts[k2] * (kUnitTiles * CG * 64) + it;
+          ulonglong2 pk = ld_packet(src);
+          if (!packet_is(pk, epoch)) pk = wait_packet(src, epoch, pp.sync, &sh->abort);
+          v0 += __uint_as_float((unsigned)pk.x);
+          v1 += __uint_as_float((unsigned)pk.y);
         }
         const int m = cg * 8 + 2 * (ln & 3) + ch;
         const int rt = grp * kUnitTiles + tile;
@@ -606,11 +633,7 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
         pp.ssq_part[grp * kPassMaxRows + tid] = s;
       }
     }
-    consumer_sync();  // red and parts may be rewritten; every thread's piece of the partial is stored
-    if (!starts_group && tid == 0) {
-      __threadfence();  // cumulative over the stores the barrier above ordered before this thread
-      st_release(pp.split_flags + cta, epoch);
-    }
+    consumer_sync();  // red and parts may be rewritten
     seg_begin = seg_end;
     seg_kt0 = 0;
     ++grp;
