@@ -58,7 +58,11 @@ constexpr int kPassMaxHeads = 48;
 constexpr int kSsqMaxGroups = 256;  // groups of 128 features of the residual stream (d_model <= 32768)
 
 enum StageKind { ST_LINEAR = 0, ST_ATTN = 1 };
-enum XMode { X_PLAIN = 0, X_ATTN_FOLD = 1 };  // how a linear stage reads its activations
+// How a linear stage reads its activations.  X_ATTN_FOLD: they are the attention output, which
+// exists only as kAttnSplits partial sums per (row, head), and every fragment load folds them.
+// X_STAGED (chosen by the kernel, never in a stage descriptor): the CTA has folded the columns
+// its units need into shared memory before its first unit.
+enum XMode { X_PLAIN = 0, X_ATTN_FOLD = 1, X_STAGED = 2 };
 enum RmsMode { RMS_NONE = 0, RMS_DIRECT = 1, RMS_FROM_PARTS = 2 };
 
 struct StageDesc {
@@ -288,10 +292,11 @@ struct XRegs {
 };
 
 struct XSource {  // the fields of the stage an activation load needs, kept in registers
-  const float* X;
+  const float* X;  // X_STAGED: shared memory, column 0 = first column of k-tile kt0
   const float* gain;
   const float* part_o;
   int ldx, n_heads;
+  int kt0, KT;  // X_STAGED only
 };
 
 // Activation fragment of k-tile kt for every column group.  X_ATTN_FOLD: the activation is the
@@ -317,6 +322,12 @@ __device__ __forceinline__ void load_xregs(XRegs<CG>& x, const XSource& xs, cons
         const float* xp = xs.X + (size_t)m * xs.ldx + kt * 16 + 2 * q;
         x.lo8[cg] = ld_act2(xp);
         x.hi8[cg] = ld_act2(xp + 8);
+      } else if (XM == X_STAGED) {
+        int dk = kt - xs.kt0;
+        if (dk < 0) dk += xs.KT;
+        const float* xp = xs.X + m * xs.ldx + dk * 16 + 2 * q;
+        x.lo8[cg] = *reinterpret_cast<const float2*>(xp);
+        x.hi8[cg] = *reinterpret_cast<const float2*>(xp + 8);
       } else {
         const int k = kt * 16 + 2 * q;
         const int head = k / HD, d = k - head * HD;
@@ -428,8 +439,60 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
     consumer_sync();
   }
 
+  // ---- or the folded activations themselves, for the k-tiles this CTA's units use ----
+  // Every element asks for its 8 (max, sum) pairs and its 8 partial values at once, so the whole
+  // fold costs one round trip to L2, where folding inside the fragment loads costs one for the
+  // weights and one more for each of the first three fragments.  Same operations in the same
+  // order as above: the result is bit-identical whichever way a CTA takes.
+  float* const x_staged = sc;  // same place: a stage uses one or the other
+  const int staged_kts = min(nun, KT), staged_ld = staged_kts * 16 + 8;  // +8: rows start 8 banks apart
+  if (XM == X_STAGED) {
+    const int n_heads = st.ep.n_heads;
+    const int pairs_per_row = staged_kts * 8;
+#pragma unroll 2
+    for (int e = tid; e < M * pairs_per_row; e += kPassConsumerThreads) {
+      const int m = e / pairs_per_row, c = (e - m * pairs_per_row) * 2;
+      int kt = kt_first + (c >> 4);
+      if (kt >= KT) kt -= KT;
+      const int k = kt * 16 + (c & 15);
+      const int head = k / HD, d = k - head * HD;
+      const size_t rh = (size_t)m * n_heads + head;
+      const float* ml = pp.part_ml + rh * kAttnSplits * 2;
+      const float* po = pp.part_o + rh * kAttnSplits * HD + d;
+      float mj[kAttnSplits], lj[kAttnSplits];
+      float2 oj[kAttnSplits];
+#pragma unroll
+      for (int j = 0; j < kAttnSplits; ++j) {
+        const float2 v = ld_act2(ml + 2 * j);
+        mj[j] = v.x;
+        lj[j] = v.y;
+        oj[j] = ld_act2(po + (size_t)j * HD);
+      }
+      float mx = -INFINITY;
+#pragma unroll
+      for (int j = 0; j < kAttnSplits; ++j)
+        if (lj[j] > 0.f) mx = fmaxf(mx, mj[j]);
+      float l = 0.f, wj[kAttnSplits];
+#pragma unroll
+      for (int j = 0; j < kAttnSplits; ++j) {
+        wj[j] = lj[j] > 0.f ? __expf(mj[j] - mx) : 0.f;
+        l = fmaf(lj[j], wj[j], l);
+      }
+      const float inv_l = l > 0.f ? 1.0f / l : 0.f;
+      float2 xv = make_float2(0.f, 0.f);
+#pragma unroll
+      for (int j = 0; j < kAttnSplits; ++j) {
+        const float w = wj[j] * inv_l;
+        xv.x = fmaf(w, oj[j].x, xv.x);
+        xv.y = fmaf(w, oj[j].y, xv.y);
+      }
+      *reinterpret_cast<float2*>(x_staged + m * staged_ld + c) = xv;
+    }
+    consumer_sync();
+  }
+
   // activation fragments of my next three units; kt_pref = k-tile of the next unit to prefetch
-  const XSource xs{st.X, st.gain, pp.part_o, st.ldx, st.ep.n_heads};
+  const XSource xs{XM == X_STAGED ? x_staged : st.X, st.gain, pp.part_o, XM == X_STAGED ? staged_ld : st.ldx, st.ep.n_heads, kt_first, KT};
   XRegs<CG> x0, x1, x2;
   int kt_pref = (kt_first + cls) % KT;
   auto prefetch = [&](XRegs<CG>& x, int i) {
@@ -981,10 +1044,21 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
       // advance by n_stages - 1 per launch, so stage s gets (bar_base + s) * 2 + (1 if it is the
       // launch's first stage): only a launch's last stage and the next launch's first would
       // otherwise collide.
-      if (sh->st.x_mode == X_PLAIN)
-        linear_stage<CG, HD, X_PLAIN>(pp, sh, ring, n_slots, work, chunk_base, 2u * ((unsigned)bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u);
-      else
-        linear_stage<CG, HD, X_ATTN_FOLD>(pp, sh, ring, n_slots, work, chunk_base, 2u * ((unsigned)bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u);
+      const unsigned serial = 2u * ((unsigned)bar_base + (unsigned)s) + (s == 0 ? 1u : 0u) + 2u;
+      if (sh->st.x_mode == X_PLAIN) {
+        linear_stage<CG, HD, X_PLAIN>(pp, sh, ring, n_slots, work, chunk_base, serial);
+      } else {
+        // fold the attention partials into shared memory first if the columns this CTA's units
+        // use fit beside the other work buffers (they do for passes of a few rows)
+        long long ub, ue;
+        unit_range((long long)sh->st.n_groups * sh->st.KT, blockIdx.x, gridDim.x, ub, ue);
+        const long long kts = ue - ub < sh->st.KT ? ue - ub : sh->st.KT;
+        const size_t need = (size_t)pp.M * (size_t)(kts * 16 + 8) * sizeof(float);
+        if (need <= pass_work_bytes<CG, HD>() - (size_t)work_sc_off<CG>())
+          linear_stage<CG, HD, X_STAGED>(pp, sh, ring, n_slots, work, chunk_base, serial);
+        else
+          linear_stage<CG, HD, X_ATTN_FOLD>(pp, sh, ring, n_slots, work, chunk_base, serial);
+      }
     } else {
       const int half = tid / kHalfThreads, htid = tid % kHalfThreads;
       const int n_heads = sh->st.ep.n_heads;
