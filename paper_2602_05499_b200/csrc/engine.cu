@@ -330,6 +330,15 @@ cudaError_t configure_pass_t(sdfp_ctx* c, int max_smem_optin) {
   if (e != cudaSuccess) return e;
   e = cudaFuncSetAttribute(pass_kernel<2, HD>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)c->pass_smem);
   if (e != cudaSuccess) return e;
+  // The kernel moves registers from its producer group to its consumers; the amounts are fixed
+  // numbers that only add up if it was compiled to the launch size they assume.  Otherwise the
+  // consumers would wait for registers that never come: refuse rather than launch.
+  for (const void* fn : {(const void*)pass_kernel<1, HD>, (const void*)pass_kernel<2, HD>}) {
+    cudaFuncAttributes fa{};
+    e = cudaFuncGetAttributes(&fa, fn);
+    if (e != cudaSuccess) return e;
+    if (fa.numRegs != kPassLaunchRegs) return cudaErrorInvalidDeviceFunction;
+  }
   // a cooperative launch needs every CTA resident at once: one per SM
   int per_sm = 0;
   e = cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, pass_kernel<2, HD>, kPassThreads, c->pass_smem);

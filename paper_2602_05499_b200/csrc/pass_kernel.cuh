@@ -45,7 +45,15 @@ namespace sdfp {
 constexpr int kClasses = 8;  // k-classes: units of a CTA's range are dealt round-robin to them
 constexpr int kPassConsumerWarps = 2 * kClasses;
 constexpr int kPassConsumerThreads = kPassConsumerWarps * 32;
-constexpr int kPassThreads = kPassConsumerThreads + 32;  // + the producer warp
+// Consumers are four warpgroups; the producer warp sits in a fifth whose other three warps only
+// give their registers away.  The kernel is launched with kPassLaunchRegs registers per thread (20
+// warps put five on every scheduler, which caps it there); the producer's group then shrinks to
+// kPassProducerRegs and every consumer grows to kPassConsumerRegs:
+// 128 * (96 - 32) = 512 * (112 - 96) registers change hands.
+constexpr int kPassThreads = kPassConsumerThreads + 128;
+constexpr int kPassLaunchRegs = 96, kPassProducerRegs = 32, kPassConsumerRegs = 112;
+static_assert(128 * (kPassLaunchRegs - kPassProducerRegs) >= kPassConsumerThreads * (kPassConsumerRegs - kPassLaunchRegs),
+              "the consumers would wait for registers nobody gives back");
 constexpr int kHalfThreads = kPassConsumerThreads / 2;   // an attention item is run by half the consumers
 constexpr int kUnitTiles = 8;                            // row tiles per unit
 constexpr int kUnitBytes = kUnitTiles * 512;
@@ -951,6 +959,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
   __syncthreads();
 
   if (tid >= kPassConsumerThreads) {
+    asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPassProducerRegs));
     // ================= producer warp: stream this CTA's share of every weight matrix =================
     if (tid == kPassConsumerThreads) {
       // Two cursors walk the same list of chunks (a chunk = up to kChunkUnits units of one stage):
@@ -1020,6 +1029,7 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
   }
 
   // ================= consumer warps =================
+  asm volatile("setmaxnreg.inc.sync.aligned.u32 %0;" ::"n"(kPassConsumerRegs));
   const unsigned long long bar_base = sh->bar_base;
   unsigned chunk_base = 0;
   bool ok = true;
