@@ -46,10 +46,10 @@ WORKLOADS = {
 SEED = 20260205
 # dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
 # capture summarised under profiles/ (null until a capture of the current kernel exists)
-# ratio measured on the 4-layer case (1075.39 MB read + 8.58 MB written against 1074.86 MB algorithmic);
+# ratio measured on the 4-layer case (1075.17 MB read + 5.72 MB written against 1074.86 MB algorithmic);
 # traffic grows in proportion to the layers a launch runs, so a full-size launch is taken as
 # ratio x its algorithmic bytes
-TRAFFIC_RATIO = 1.0085
+TRAFFIC_RATIO = 1.0056
 PAPER_CONTEXT = "paper reports 1.32x-1.5x over vanilla decoding for LLaMA-2-13B/70B on unstated hardware"
 
 
