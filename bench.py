@@ -36,17 +36,22 @@ import synth_inputs as si  # noqa: E402
 
 METRIC = "decode tokens/s (batch 1, 7B-shape bf16), speedup vs AR decode, HBM % roofline"
 WORKLOADS = {
-    # name: (shape, n_skip, k, prompt_len, max_new, temperature)
-    "c2-7b-greedy-k4": (si.LLAMA7B, 12, 4, 512, 256, 0.0),       # the configuration the metric is quoted on
-    "c3-7b-sampled-k6": (si.LLAMA7B, 12, 6, 512, 256, 1.0),      # rejection sampling, residual resampling
-    "c4-13b-greedy-k4": (si.LLAMA13B, 16, 4, 2048, 512, 0.0),    # long KV cache
-    "c1-tiny-greedy-k4": (si.TINY, 2, 4, 16, 64, 0.0),
-    "7b-4layers-greedy-k4": (si.LLAMA7B_4L, 2, 4, 64, 64, 0.0),
+    # name: (shape, n_skip, k, prompt_len, max_new, temperature, batch)
+    "c2-7b-greedy-k4": (si.LLAMA7B, 12, 4, 512, 256, 0.0, 1),       # the configuration the metric is quoted on
+    "c3-7b-sampled-k6": (si.LLAMA7B, 12, 6, 512, 256, 1.0, 1),      # rejection sampling, residual resampling
+    "c4-13b-greedy-k4": (si.LLAMA13B, 16, 4, 2048, 512, 0.0, 1),    # long KV cache
+    "c1-tiny-greedy-k4": (si.TINY, 2, 4, 16, 64, 0.0, 1),
+    "7b-4layers-greedy-k4": (si.LLAMA7B_4L, 2, 4, 64, 64, 0.0, 1),
+    "7b-4layers-b8-greedy-k4": (si.LLAMA7B_4L, 2, 4, 64, 64, 0.0, 8),
 }
+# batch 8 with ragged acceptance: draft length k and share of skipped layers swept
+for _k in (2, 4, 8):
+    for _skip in (8, 12, 16):
+        WORKLOADS["c5-7b-b8-greedy-k%d-skip%d" % (_k, _skip)] = (si.LLAMA7B, _skip, _k, 1024, 256, 0.0, 8)
 SEED = 20260205
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel, from the ncu
-# capture summarised under profiles/ (null until a capture of the current kernel exists)
-# ratio measured on the 4-layer case (1075.17 MB read + 5.72 MB written against 1074.86 MB algorithmic);
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the dominant kernel against its
+# algorithmic bytes, from an ncu capture of the kernel as it stands (None when there is none):
+# measured on the 4-layer case (1075.17 MB read + 5.72 MB written against 1074.86 MB algorithmic);
 # traffic grows in proportion to the layers a launch runs, so a full-size launch is taken as
 # ratio x its algorithmic bytes
 TRAFFIC_RATIO = 1.0056
@@ -161,7 +166,7 @@ def reduce_over_ranks(times, counts, device, world):
 def run_reference(args, workload):
     """--impl reference: the oracle on the host cores (rank 0 only)."""
     import torch
-    shape, n_skip, k, plen, n_new, temp = WORKLOADS[workload]
+    shape, n_skip, k, plen, n_new, temp, _batch = WORKLOADS[workload]
     skip = si.choose_skip_layers(shape.n_layers, n_skip)
     cores = os.cpu_count() or 1
     big = shape.n_params() > 1e9
@@ -195,7 +200,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2-7b-greedy-k4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
-    ap.add_argument("--flags", type=int, default=0, help="sdfp_config.flags (1 no graph, 2 no PDL, 4 FMA GEMM)")
+    ap.add_argument("--flags", type=int, default=0, help="sdfp_config.flags (1 no graph, 2 no PDL, 4 FMA GEMM, 8 one kernel per operation instead of the whole-pass kernel)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
@@ -218,17 +223,17 @@ def main():
         dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
     pkg.build_library()
 
-    shape, n_skip, k, plen, n_new, temp = WORKLOADS[args.workload]
+    shape, n_skip, k, plen, n_new, temp, batch = WORKLOADS[args.workload]
     skip = si.choose_skip_layers(shape.n_layers, n_skip)
     dev = f"cuda:{local_rank}"
     w = si.make_weights(shape, skip, device=dev)
-    eng = pkg.Sdfp(shape, w, max_seq=plen + n_new + 16, max_batch=1, k_max=8, flags=args.flags)
+    eng = pkg.Sdfp(shape, w, max_seq=plen + n_new + 16, max_batch=batch, k_max=8, flags=args.flags)
     eng.sdfp_set_draft_layers(si.keep_mask(shape.n_layers, skip))
     want_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
     w_cpu = si.weights_to(w, "cpu") if want_cpu else None
     del w
     torch.cuda.empty_cache()
-    prompts = si.make_prompts(shape.vocab, 1, plen, seed=si.PROMPT_SEED + 1000 * rank)
+    prompts = si.make_prompts(shape.vocab, batch, plen, seed=si.PROMPT_SEED + 1000 * rank)
 
     def barrier():
         if world > 1:
@@ -278,7 +283,7 @@ def main():
     for _ in range(ar_steps):
         ar = eng.sdfp_generate(prompts, 0, n_new, temp, SEED)
         ar_dec_ms += ar.timing["decode_ms"]
-    ar_tok_s = ar_steps * n_new / (ar_dec_ms * 1e-3)
+    ar_tok_s = ar_steps * batch * n_new / (ar_dec_ms * 1e-3)
     ar_t = ar.timing
     ar_pass_gbs = (ar_t["weight_bytes"] + ar_t["kv_bytes"]) / (ar_t["decode_ms"] * 1e-3) / 1e9
     if temp == 0.0:
@@ -290,7 +295,8 @@ def main():
     peak, peak_src = measured_peak_gbs()
     per_kernel = {}
     mid = plen + n_new // 2                      # a context in the middle of the generation
-    uses_pass = shape.dtype == "bf16" and not (args.flags & (pkg.FLAG_NO_PASS_KERNEL | pkg.FLAG_FMA_GEMM))
+    uses_pass = (shape.dtype == "bf16" and not (args.flags & (pkg.FLAG_NO_PASS_KERNEL | pkg.FLAG_FMA_GEMM))
+                 and batch * 9 <= 16)          # k_max = 8: wider contexts run one kernel per operation
     if uses_pass:
         for name, draft, rows in (("draft_pass@M=1", True, 1), ("draft_pass@M=2", True, 2),
                                   ("verify_pass@M=%d" % (k + 1), False, k + 1), ("ar_pass@M=1", False, 1)):
@@ -302,12 +308,12 @@ def main():
             shape.n_layers - len(skip), shape.n_layers, mid)
     else:
         names = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
-        for rows in (1, k + 1):
+        for rows in (batch, batch * (k + 1)):
             for which, nm in enumerate(names):
                 ms, nbytes = eng.sdfp_time_linear(which, rows, 64 if which < 4 else 16)
                 per_kernel[f"{nm}@M={rows}"] = {"us": round(ms * 1e3, 2), "GB/s": round(nbytes / ms / 1e6, 1)}
-        dom_ms, dom_bytes = eng.sdfp_time_linear(2, k + 1, 128)
-        dom_name = "linear kernel (gate/up, M=%d)" % (k + 1)
+        dom_ms, dom_bytes = eng.sdfp_time_linear(2, batch * (k + 1), 128)
+        dom_name = "linear kernel (gate/up, M=%d)" % (batch * (k + 1))
     kernel_gbs = dom_bytes / dom_ms / 1e6
 
     # ---- reduce over ranks --------------------------------------------------------------------------
@@ -332,7 +338,7 @@ def main():
             "metric": METRIC, "value": value, "unit": "tokens/s", "n_gpus": world, "steps": args.steps,
             "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32", "data": "synthetic",
-            "config": {"workload": args.workload, "shape": shape.name, "batch": 1, "prompt_len": plen,
+            "config": {"workload": args.workload, "shape": shape.name, "batch": batch, "prompt_len": plen,
                        "max_new": n_new, "k": k, "skip_layers": skip,
                        "decoding": "greedy" if temp == 0.0 else "sampled, temperature %g, Philox seed %d" % (temp, SEED),
                        "l2": "inputs larger than L2 (weights %.1f GB per pass)" % (shape.n_params() * 2 / 1e9)
@@ -343,7 +349,7 @@ def main():
             "acceptance_rate": float(np.mean(acc)), "tokens_per_round": float(np.mean(tau)),
             "prefill_ms_per_step": pre_ms / args.steps,
             "e2e": {"value": e2e_value, "unit": "tokens/s", "h2d_bytes_per_step": int(prompts.nbytes),
-                    "d2h_bytes_per_step": int(4 * n_new + 4 + 12 * (n_new + 1)),
+                    "d2h_bytes_per_step": int(batch * (4 * n_new + 4 + 12 * (n_new + 1))),
                     "note": "whole sdfp_generate call: prompt copy, prefill of both caches, decode, token copy"},
             "gpu_launches": int(launches_all),
             "clocks": clocks,

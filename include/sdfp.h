@@ -19,7 +19,16 @@
  *     caller keeps ownership; NULL = the legacy default stream).
  *   - Deterministic: same config, weights, mask, prompts, k, temperature and
  *     seed give bit-identical outputs, and a sequence's tokens do not depend on
- *     what else is in the batch nor on how many rows a pass carries.
+ *     what else is in the batch nor on how many rows a pass carries.  (A context
+ *     takes one arithmetic path for all its passes: bf16 contexts whose widest
+ *     pass, max_batch*max(k_max+1, 2) rows, fits 16 rows run every pass in the
+ *     persistent whole-pass kernel, all others run one kernel per operation.)
+ *   - A context belongs to the device that was current at sdfp_create; calls made
+ *     with another device current fail with SDFP_ESTATE before touching the GPU.
+ *   - Kernels that wait on one another (the whole-pass kernel's grid barriers and
+ *     hand-offs) bound every wait; a wait that runs out ends the call with
+ *     SDFP_ETIMEOUT, the outputs of that call are invalid, and the context can be
+ *     used again.
  *   - There is no CPU fallback: without a usable CUDA device every entry point
  *     that computes fails with SDFP_ECUDA.
  */
@@ -40,7 +49,8 @@ typedef enum {
   SDFP_EINVAL = -1, /* bad argument or unsupported shape            */
   SDFP_ENOMEM = -2, /* device or host allocation failed             */
   SDFP_ECUDA = -3,  /* a CUDA call failed (text in sdfp_last_error) */
-  SDFP_ESTATE = -4  /* call not valid in the context's state        */
+  SDFP_ESTATE = -4, /* call not valid in the context's state        */
+  SDFP_ETIMEOUT = -5 /* a bounded wait inside a kernel ran out; the context stays usable */
 } sdfp_status;
 
 typedef enum { SDFP_F32 = 0, SDFP_BF16 = 1 } sdfp_dtype;
@@ -58,7 +68,8 @@ typedef enum { SDFP_F32 = 0, SDFP_BF16 = 1 } sdfp_dtype;
  * embeddings on pairs (i, i + head_dim/2) with base rope_theta, multi-head
  * causal attention (n_kv_heads == n_heads), SwiGLU FFN, untied lm-head, no bias.
  * Requirements: d_model == n_heads*head_dim; head_dim in {64, 128}; d_model,
- * d_ffn and vocab multiples of 16; max_batch*(k_max+1) <= 64.
+ * d_ffn and vocab multiples of 16; max_batch <= 16, k_max <= 15 and
+ * max_batch*max(k_max+1, 2) <= 80 rows per pass (8 sequences with k = 8: 72).
  */
 typedef struct {
   int32_t n_layers, d_model, n_heads, head_dim, d_ffn, vocab;
@@ -155,7 +166,7 @@ int sdfp_generate(sdfp_ctx *ctx, const int32_t *prompts, int32_t batch, int32_t 
  * Test hook: run `rows` tokens of ONE sequence at positions start.. through the
  * target (draft == 0) or the draft (draft != 0) model on sequence slot 0,
  * writing K/V into that model's cache from `start` on, and copy the logits
- * [rows, vocab] (fp32) to host.  rows <= 64.  Lets a test compare logits with
+ * [rows, vocab] (fp32) to host.  rows <= 80.  Lets a test compare logits with
  * the oracle position by position, in chunks of any size.
  */
 int sdfp_forward_logits(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int32_t rows,
@@ -186,7 +197,8 @@ int sdfp_forward_logits(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int
  *     16) and P = ceil((start + rows) / 64).  The message states both sizes.
  *   - The first call on a device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and keeps it.  Make that first call
- *     before starting any stream capture.
+ *     before starting any stream capture, and from one thread: two threads making the first
+ *     call on a device at the same time both store the (same) address without synchronisation.
  *   - All contexts of the process on one device share the array, and it keeps what the last
  *     call left in it.  The call clears the part that must start at zero itself, but two such
  *     calls whose GPU work overlaps (different streams, different threads) race on it:
@@ -224,6 +236,17 @@ int sdfp_time_linear(sdfp_ctx *ctx, int32_t which, int32_t rows, int32_t iters,
  */
 int sdfp_time_pass(sdfp_ctx *ctx, int32_t draft, int32_t rows, int32_t position, int32_t iters,
                    float *ms_per_launch, int64_t *bytes_per_launch);
+
+/*
+ * Failure-path test hook (whole-pass kernel contexts; SDFP_ESTATE otherwise).  Section II-A's
+ * loop has no counterpart: this exercises the library's own bounded waits.  After the call,
+ * the grid barriers of the next pass expect one arrival more than the grid can provide and
+ * every wait gives up after wait_limit_ns (1 ms .. 2 s) instead of the default 2 s: that pass
+ * winds down in an orderly way (nothing faults, nothing spins on), the entry point that
+ * launched it returns SDFP_ETIMEOUT with the name of the wait in sdfp_last_error, and in
+ * doing so puts barrier and limit back to normal, so the next call on the context works.
+ */
+int sdfp_debug_expire_next_wait(sdfp_ctx *ctx, uint64_t wait_limit_ns);
 
 const char *sdfp_last_error(const sdfp_ctx *ctx);
 void sdfp_destroy(sdfp_ctx *ctx);

@@ -16,7 +16,8 @@ SDFP_F32, SDFP_BF16 = 0, 1
 FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_FMA_GEMM, FLAG_NO_PASS_KERNEL = 1, 2, 4, 8
 
 EXPORTS = ["sdfp_create", "sdfp_set_draft_layers", "sdfp_generate", "sdfp_forward_logits",
-           "sdfp_forward_logits_static", "sdfp_get_timing", "sdfp_time_linear", "sdfp_time_pass", "sdfp_last_error", "sdfp_destroy"]
+           "sdfp_forward_logits_static", "sdfp_get_timing", "sdfp_time_linear", "sdfp_time_pass",
+           "sdfp_debug_expire_next_wait", "sdfp_last_error", "sdfp_destroy"]
 
 
 class SdfpConfig(C.Structure):
@@ -87,6 +88,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdfp_time_pass.argtypes = [vp, C.c_int32, C.c_int32, C.c_int32, C.c_int32, C.POINTER(C.c_float),
                                    C.POINTER(C.c_int64)]
     lib.sdfp_time_pass.restype = C.c_int
+    lib.sdfp_debug_expire_next_wait.argtypes = [vp, C.c_uint64]
+    lib.sdfp_debug_expire_next_wait.restype = C.c_int
     lib.sdfp_last_error.argtypes = [vp]
     lib.sdfp_last_error.restype = C.c_char_p
     lib.sdfp_destroy.argtypes = [vp]
@@ -220,6 +223,9 @@ class Sdfp:
         nbytes = C.c_int64(0)
         self._check(self.lib.sdfp_time_linear(self.handle, which, rows, iters, C.byref(ms), C.byref(nbytes)))
         return ms.value, nbytes.value
+
+    def sdfp_debug_expire_next_wait(self, wait_limit_ns: int):
+        self._check(self.lib.sdfp_debug_expire_next_wait(self.handle, C.c_uint64(wait_limit_ns)))
 
     def sdfp_time_pass(self, draft: bool, rows: int, position: int, iters: int):
         """(ms per launch of the whole-pass kernel, bytes such a launch has to move)."""

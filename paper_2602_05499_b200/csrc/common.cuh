@@ -7,7 +7,7 @@
 
 namespace sdfp {
 
-constexpr int kMaxRows = 64;    // rows (tokens) one pass may carry
+constexpr int kMaxRows = 80;    // rows (tokens) one pass may carry: 8 sequences x (k = 8 drafts + 1) = 72, in column groups of 8
 constexpr int kAttnChunk = 64;  // keys per attention work unit; fixed so that a
                                 // row's result never depends on the context length
                                 // of other rows or on how many rows share the sweep

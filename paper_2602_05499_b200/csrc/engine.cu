@@ -57,6 +57,7 @@ struct sdfp_ctx {
   bool bf16 = false, use_mma = false, use_pdl = true, use_graph = true;
   size_t esz = 4;  // bytes per stored element
   int num_sms = 148;
+  int device = -1;  // ordinal that was current at sdfp_create; every computing call checks it is still current
 
   std::vector<LayerWeights> layers;
   void* embed = nullptr;
@@ -118,6 +119,20 @@ int fail(sdfp_ctx* c, int code, const char* fmt, ...) {
   else
     g_create_error = buf;
   return code;
+}
+
+// The context's memory, stream and kernels belong to the device that was current at sdfp_create.
+// With another device current a launch on the legacy default stream (or a symbol lookup) would land
+// on the wrong GPU, so every entry point that touches the device checks first.
+int check_device(sdfp_ctx* c, const char* who) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) {
+    cudaGetLastError();
+    return fail(c, SDFP_ECUDA, "%s: cudaGetDevice failed", who);
+  }
+  if (dev != c->device)
+    return fail(c, SDFP_ESTATE, "%s: the context was created on device %d but device %d is current", who, c->device, dev);
+  return 0;
 }
 
 #define CU_OK(c, call)                                                                          \
@@ -228,8 +243,7 @@ cudaError_t configure_kernels(const sdfp_ctx* c) {
     e = hd128 ? configure_attention_t<__nv_bfloat16, 128>() : configure_attention_t<__nv_bfloat16, 64>();
   else
     e = hd128 ? configure_attention_t<float, 128>() : configure_attention_t<float, 64>();
-  if (e != cudaSuccess) return e;
-  return configure_linear_mma();
+  return e;
 }
 
 // ---- persistent pass kernel: stage lists and launch ---------------------------------------------
@@ -412,7 +426,8 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
                     (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
                     reinterpret_cast<const float*>(c->embed), c->h, d));
   const KvCache& kv = draft ? c->cache_d : c->cache_t;
-  const bool whole_pass = c->use_pass && rows <= kPassMaxRows;
+  const bool whole_pass = c->use_pass;  // a context takes ONE path for all its passes (see sdfp_create)
+  if (whole_pass && rows > kPassMaxRows) return fail(c, SDFP_ESTATE, "a pass of %d rows reached the whole-pass kernel", rows);
   if (whole_pass) CU_OK(c, run_pass(c, draft, rows, attn_rows_per_seq, decide != DECIDE_NONE));
   for (int l = 0; l < g.n_layers && !whole_pass; ++l) {
     if (draft && !c->keep[l]) continue;  // Algorithm 1: pruned layers are removed from the draft
@@ -470,13 +485,14 @@ int enqueue_round(sdfp_ctx* c, int k, int batch, bool sampled, int n_chunks) {
   pd.rows_per_seq = k + 1;
   if (int r = enqueue_pass(c, pd, false, (k + 1) * batch, k + 1, n_chunks, sampled ? DECIDE_LOGITS : DECIDE_ARGMAX))
     return r;
+  const int* pass_err = c->use_pass ? &c->psync->error : nullptr;
   if (sampled)
     CU_OK(c, launch(c, accept_sampled_kernel, dim3(1), dim3(kSampleThreads), 0, c->gs, (const float*)c->logits,
                     c->cfg.vocab, (const int*)c->draft_tok, (const float*)c->qprob, (const double*)c->qsum, c->seq_tok,
-                    c->cfg.max_seq, c->out_tok, c->stats));
+                    c->cfg.max_seq, c->out_tok, c->stats, pass_err));
   else
     CU_OK(c, launch(c, accept_greedy_kernel, dim3(1), dim3(32), 0, c->gs, (const int*)c->draft_tok,
-                    (const int*)c->tgt_tok, c->seq_tok, c->cfg.max_seq, c->out_tok, c->stats));
+                    (const int*)c->tgt_tok, c->seq_tok, c->cfg.max_seq, c->out_tok, c->stats, pass_err));
   return 0;
 }
 
@@ -592,7 +608,8 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   if (g.max_batch < 1 || g.max_batch > kMaxBatch) return fail(nullptr, SDFP_EINVAL, "max_batch must be 1..%d", kMaxBatch);
   if (g.k_max < 0 || g.k_max > kMaxK) return fail(nullptr, SDFP_EINVAL, "k_max must be 0..%d", kMaxK);
   if (g.max_batch * (g.k_max + 1) > kMaxRows || g.max_batch * 2 > kMaxRows)
-    return fail(nullptr, SDFP_EINVAL, "max_batch*(k_max+1) must not exceed %d", kMaxRows);
+    return fail(nullptr, SDFP_EINVAL, "max_batch*(k_max+1) = %d exceeds the %d rows a pass can carry",
+                g.max_batch * std::max(g.k_max + 1, 2), kMaxRows);
   if (g.max_seq < 4 || !(g.rms_eps > 0.f) || !(g.rope_theta > 0.f)) return fail(nullptr, SDFP_EINVAL, "bad max_seq, rms_eps or rope_theta");
   if (!w->tok_embed || !w->final_norm || !w->lm_head || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up ||
       !w->w_down || !w->attn_norm || !w->ffn_norm)
@@ -641,9 +658,16 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
     return bail(SDFP_ECUDA);
   }
   c->num_sms = prop.multiProcessorCount;
+  c->device = dev;
+  // One arithmetic path per context.  The whole-pass kernel and the per-operation kernels add a
+  // dot product's terms in different orders, so a context whose widest pass (a verify pass of
+  // max_batch sequences, or the two-row draft pass) does not fit the whole-pass kernel runs
+  // every pass, narrow ones included, on the per-operation kernels: only then is a row's
+  // result independent of the pass it sits in, and speculative output equal to autoregressive
+  // output bit for bit.
+  const int widest = g.max_batch * std::max(g.k_max + 1, 2);
   c->use_pass = c->use_mma && !(g.flags & SDFP_FLAG_NO_PASS_KERNEL) && prop.cooperativeLaunch && g.d_model >= 64 &&
-
-                g.n_heads <= kPassMaxHeads && g.d_model / 128 + 1 <= kSsqMaxGroups;
+                g.n_heads <= kPassMaxHeads && g.d_model / 128 + 1 <= kSsqMaxGroups && widest <= kPassMaxRows;
   if (c->use_pass) {
     int optin = 0;
     cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
@@ -726,6 +750,7 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
 extern "C" int sdfp_set_draft_layers(sdfp_ctx* c, const uint8_t* keep_mask) {
   if (!c) return SDFP_EINVAL;
   if (!keep_mask) return fail(c, SDFP_EINVAL, "keep_mask is NULL");
+  if (int r = check_device(c, "sdfp_set_draft_layers")) return r;
   int kept = 0;
   for (int l = 0; l < c->cfg.n_layers; ++l) kept += keep_mask[l] ? 1 : 0;
   if (kept == 0) return fail(c, SDFP_EINVAL, "the draft must keep at least one layer");
@@ -756,7 +781,7 @@ int check_pass_error(sdfp_ctx* c) {
   cudaStreamSynchronize(c->stream);
   static const char* const what[] = {"", "grid barrier", "weight slot never filled", "weight slot never freed",
                                      "partial sum of a split group never posted"};
-  return fail(c, SDFP_ECUDA, "pass kernel gave up a wait (%s); results of this call are invalid",
+  return fail(c, SDFP_ETIMEOUT, "pass kernel gave up a wait (%s); results of this call are invalid",
               ps.error >= 1 && ps.error <= 4 ? what[ps.error] : "unknown");
 }
 
@@ -816,6 +841,7 @@ extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch,
   if (!c) return SDFP_EINVAL;
   const sdfp_config& g = c->cfg;
   if (!prompts || !out_tokens || !out_len) return fail(c, SDFP_EINVAL, "sdfp_generate: NULL pointer");
+  if (int r = check_device(c, "sdfp_generate")) return r;
   if (batch < 1 || batch > g.max_batch) return fail(c, SDFP_EINVAL, "batch %d outside 1..%d", batch, g.max_batch);
   if (k < 0 || k > g.k_max) return fail(c, SDFP_EINVAL, "k %d outside 0..%d", k, g.k_max);
   if (prompt_len < 1 || max_new < 1) return fail(c, SDFP_EINVAL, "prompt_len and max_new must be >= 1");
@@ -897,9 +923,9 @@ extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch,
       return r;
     }
     ++rounds;
-    CU_OK(c, cudaMemcpyAsync(c->pinned_flag, &c->gs->all_done, 4, cudaMemcpyDeviceToHost, st));
+    CU_OK(c, cudaMemcpyAsync(c->pinned_flag, &c->gs->all_done, 8, cudaMemcpyDeviceToHost, st));  // all_done, pass_error
     CU_OK(c, cudaStreamSynchronize(st));
-    if (c->pinned_flag[0]) break;
+    if (c->pinned_flag[0] || c->pinned_flag[1]) break;
   }
   CU_OK(c, cudaEventRecord(c->ev[2], st));
   if (int r = check_pass_error(c)) return r;
@@ -954,6 +980,7 @@ extern "C" int sdfp_forward_logits(sdfp_ctx* c, int32_t draft, const int32_t* to
   if (!c) return SDFP_EINVAL;
   const sdfp_config& g = c->cfg;
   if (!tokens || !host_logits) return fail(c, SDFP_EINVAL, "sdfp_forward_logits: NULL pointer");
+  if (int r = check_device(c, "sdfp_forward_logits")) return r;
   if (rows < 1 || rows > kMaxRows) return fail(c, SDFP_EINVAL, "rows %d outside 1..%d", rows, kMaxRows);
   if (start < 0 || start + rows > g.max_seq) return fail(c, SDFP_EINVAL, "positions exceed max_seq");
   for (int i = 0; i < rows; ++i)
@@ -979,8 +1006,7 @@ void* g_static_scratch_addr[kMaxDevices] = {};  // device address of the array, 
 // In host code `g_static_scratch` is only a handle for the symbol; the address a kernel can
 // use has to be asked for, once per device, with that device current.
 int static_scratch_address(sdfp_ctx* c, unsigned char** out) {
-  int dev = -1;
-  CU_OK(c, cudaGetDevice(&dev));
+  const int dev = c->device;  // current: the caller checked
   if (dev < 0 || dev >= kMaxDevices) return fail(c, SDFP_ECUDA, "device ordinal %d not supported", dev);
   if (!g_static_scratch_addr[dev]) {
     void* p = nullptr;
@@ -1001,6 +1027,7 @@ extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int3
   if (!c) return SDFP_EINVAL;
   const sdfp_config& g = c->cfg;
   if (!tokens || !host_logits) return fail(c, SDFP_EINVAL, "sdfp_forward_logits_static: NULL pointer");
+  if (int r = check_device(c, "sdfp_forward_logits_static")) return r;
   if (rows < 1 || rows > kMaxRows) return fail(c, SDFP_EINVAL, "rows %d outside 1..%d", rows, kMaxRows);
   if (start < 0 || start + rows > g.max_seq) return fail(c, SDFP_EINVAL, "positions exceed max_seq");
   for (int i = 0; i < rows; ++i)
@@ -1039,6 +1066,18 @@ extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int3
   return r;
 }
 
+extern "C" int sdfp_debug_expire_next_wait(sdfp_ctx* c, uint64_t wait_limit_ns) {
+  if (!c) return SDFP_EINVAL;
+  if (int r = check_device(c, "sdfp_debug_expire_next_wait")) return r;
+  if (!c->use_pass) return fail(c, SDFP_ESTATE, "sdfp_debug_expire_next_wait: this context does not use the whole-pass kernel");
+  if (wait_limit_ns < 1000000ull || wait_limit_ns > 2000000000ull)
+    return fail(c, SDFP_EINVAL, "sdfp_debug_expire_next_wait: the limit must lie between 1 ms and 2 s");
+  const unsigned long long words[2] = {1ull, (unsigned long long)wait_limit_ns};  // bar_extra, wait_limit_ns
+  CU_OK(c, cudaMemcpyAsync(&c->psync->bar_extra, words, sizeof words, cudaMemcpyHostToDevice, c->stream));
+  CU_OK(c, cudaStreamSynchronize(c->stream));  // words is a local
+  return 0;
+}
+
 extern "C" int sdfp_get_timing(const sdfp_ctx* c, sdfp_timing* out) {
   if (!c || !out) return SDFP_EINVAL;
   *out = c->timing;
@@ -1050,6 +1089,7 @@ extern "C" int sdfp_time_pass(sdfp_ctx* c, int32_t draft, int32_t rows, int32_t 
   if (!c) return SDFP_EINVAL;
   const sdfp_config& g = c->cfg;
   if (!ms_per_launch || !bytes_per_launch) return fail(c, SDFP_EINVAL, "sdfp_time_pass: NULL pointer");
+  if (int r = check_device(c, "sdfp_time_pass")) return r;
   if (!c->use_pass) return fail(c, SDFP_ESTATE, "sdfp_time_pass: this context does not use the whole-pass kernel");
   if (rows < 1 || rows > kPassMaxRows || iters < 1 || iters > 256 || position < 0 || position + rows > g.max_seq)
     return fail(c, SDFP_EINVAL, "sdfp_time_pass: bad argument");
@@ -1061,13 +1101,14 @@ extern "C" int sdfp_time_pass(sdfp_ctx* c, int32_t draft, int32_t rows, int32_t 
   pd.count = rows;
   pd.src = c->fwd_tok;
   std::vector<cudaEvent_t> ev(2 * (size_t)iters, nullptr);
-  for (auto& e : ev) CU_OK(c, cudaEventCreate(&e));
+  cudaError_t err = cudaSuccess;
+  for (auto& e : ev)
+    if (err == cudaSuccess) err = cudaEventCreate(&e);  // on failure the loops below do nothing and every event made so far is destroyed
   auto plan = [&]() -> cudaError_t {
     return launch(c, plan_embed_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs,
                   (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
                   reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, g.d_model);
   };
-  cudaError_t err = cudaSuccess;
   for (int i = 0; i < 3 && err == cudaSuccess; ++i) {  // warm-up
     err = plan();
     if (err == cudaSuccess) err = run_pass(c, draft != 0, rows, rows, true);
@@ -1085,7 +1126,8 @@ extern "C" int sdfp_time_pass(sdfp_ctx* c, int32_t draft, int32_t rows, int32_t 
     err = cudaEventElapsedTime(&ms, ev[2 * i], ev[2 * i + 1]);
     total += ms;
   }
-  for (auto& e : ev) cudaEventDestroy(e);
+  for (auto& e : ev)
+    if (e) cudaEventDestroy(e);
   CU_OK(c, err);
   if (int r = check_pass_error(c)) return r;
   *ms_per_launch = (float)(total / iters);
@@ -1101,6 +1143,7 @@ extern "C" int sdfp_time_linear(sdfp_ctx* c, int32_t which, int32_t rows, int32_
   if (!c) return SDFP_EINVAL;
   const sdfp_config& g = c->cfg;
   if (!ms_per_launch || !weight_bytes_per_launch) return fail(c, SDFP_EINVAL, "sdfp_time_linear: NULL pointer");
+  if (int r = check_device(c, "sdfp_time_linear")) return r;
   if (which < 0 || which > 4 || rows < 1 || rows > kMaxRows || iters < 1)
     return fail(c, SDFP_EINVAL, "sdfp_time_linear: bad argument");
   const int d = g.d_model, f = g.d_ffn;

@@ -1,7 +1,7 @@
 // Tensor-core weight-streaming linear kernel for bf16 models:
 //   Y[m, n] = Σ_k W[n, k] · X'[m, k]   with X' = X or g ⊙ X / rms(X)   (+ fused epilogue).
 //
-// The work is bound by the bytes of W (each weight is used for at most 64 rows), so the
+// The work is bound by the bytes of W (each weight is used for at most 80 rows), so the
 // kernel is organised around the weight stream, not around the MMA:
 //   * W is re-packed once into 16x16 tiles in the register order of the A operand of
 //     mma.sync.m16n8k16 (out-features on the 16-row side), 512 contiguous bytes per tile,
@@ -29,7 +29,6 @@
 
 namespace sdfp {
 
-constexpr bool kHaveMma = true;
 constexpr int kMmaThreads = 256;
 constexpr int kMmaWarps = 8;
 
@@ -216,8 +215,6 @@ inline cudaError_t launch_mma_t(const Launcher& L, const void* W, const float* X
                        reinterpret_cast<const uint4*>(W), X, ldx, M, K, NT, gain, eps, ep);
 }
 
-inline cudaError_t configure_linear_mma() { return cudaSuccess; }
-
 // n_pairs = out_features / 2; W in the tile order written by pack_mma.
 inline cudaError_t launch_linear_mma(const Launcher& L, int num_sms, const void* W, const float* X, int ldx, int M, int K,
                                      int n_pairs, const float* gain, float eps, const EpiParams& ep) {
@@ -236,7 +233,8 @@ inline cudaError_t launch_linear_mma(const Launcher& L, int num_sms, const void*
     if ((NT + 1) / 2 >= want) return launch_mma_t<2, 4, 1>(L, W, X, ldx, M, K, NT, gain, eps, ep);
     return launch_mma_t<1, 4, 2>(L, W, X, ldx, M, K, NT, gain, eps, ep);
   }
-  return launch_mma_t<1, 8, 1>(L, W, X, ldx, M, K, NT, gain, eps, ep);
+  if (M <= 64) return launch_mma_t<1, 8, 1>(L, W, X, ldx, M, K, NT, gain, eps, ep);
+  return launch_mma_t<1, 10, 1>(L, W, X, ldx, M, K, NT, gain, eps, ep);
 }
 
 }  // namespace sdfp

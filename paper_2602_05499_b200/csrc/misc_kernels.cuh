@@ -16,6 +16,7 @@ struct GenState {
   int done[kMaxBatch];
   int round;
   int all_done;
+  int pass_error;  // directly after all_done: the host reads both with one copy per round
   // parameters of the running sdfp_generate call
   int batch, k, max_new, eos_id, max_rounds;
   float temperature;
@@ -183,7 +184,7 @@ __device__ __forceinline__ void commit_tokens(volatile GenState* gs, int b, int 
 // plain autoregressive step.
 __global__ void __launch_bounds__(32)
 accept_greedy_kernel(GenState* gs_, const int* draft_tok, const int* tgt_tok, int* seq_tok, int max_seq,
-                     int* out_tok, RoundStat* stats) {
+                     int* out_tok, RoundStat* stats, const int* pass_error) {
   volatile GenState* gs = gs_;
   pdl_wait();
   pdl_launch_dependents();
@@ -206,6 +207,7 @@ accept_greedy_kernel(GenState* gs_, const int* draft_tok, const int* tgt_tok, in
   if (threadIdx.x == 0) {
     gs->round += 1;
     gs->all_done = all ? 1 : 0;
+    gs->pass_error = pass_error ? ld_act(pass_error) : 0;  // a pass of this round gave up a wait
   }
 }
 

@@ -94,6 +94,12 @@ struct PassSync {                // one per context, in global memory, zero-init
   unsigned pad0[30];
   int error;           // first PassError seen, sticky
   unsigned pad1[31];
+  // Failure-path test hook, both zero in normal operation: every grid barrier expects this many
+  // arrivals more than the grid provides (so its wait can only run out), and waits give up after
+  // wait_limit_ns nanoseconds instead of the default (0 = default).
+  unsigned long long bar_extra;
+  unsigned long long wait_limit_ns;
+  unsigned pad2[28];
 };
 
 struct PassParams {
@@ -210,6 +216,7 @@ struct PassShared {
   float inv_rms[kPassMaxRows];
   int row_pos[kPassMaxRows], row_seq[kPassMaxRows];  // fixed for the whole pass
   unsigned long long bar_base;
+  unsigned long long bar_extra;  // PassSync::bar_extra as found at launch
   int abort;     // set by whichever thread gives up a wait
   int decision;  // abort as sampled by thread 0 between two consumer barriers: uniform for all
   float attn_m[2][kPassAttnR], attn_l[2][kPassAttnR], attn_a[2][kPassAttnR];
@@ -241,7 +248,8 @@ __device__ __forceinline__ bool bounded_wait(Pred pred, PassSync* sync, volatile
         *s_abort = 1;
         return false;
       }
-      if (global_ns() - t0 > kWaitLimitNs) {
+      const unsigned long long set = *reinterpret_cast<volatile unsigned long long*>(&sync->wait_limit_ns);
+      if (global_ns() - t0 > (set ? set : kWaitLimitNs)) {
         atomicCAS(&sync->error, 0, code);
         *s_abort = 1;
         return false;
@@ -276,7 +284,7 @@ __device__ __noinline__ ulonglong2 wait_packet(const ulonglong2* src, unsigned s
 __device__ __forceinline__ bool grid_barrier(PassSync* sync, unsigned long long serial, PassShared* sh) {
   consumer_sync();
   if (threadIdx.x == 0) {
-    const unsigned long long target = serial * gridDim.x;
+    const unsigned long long target = serial * gridDim.x + sh->bar_extra;
     __threadfence();
     red_add_relaxed(&sync->bar_count, 1ull);
     bounded_wait([&] { return ld_relaxed(&sync->bar_count) >= target; }, sync, &sh->abort, PASS_ERR_GRID_BARRIER);
@@ -945,18 +953,24 @@ __global__ void __launch_bounds__(kPassThreads, 1) pass_kernel(PassParams pp, in
       mbar_init(&sh->full[s], 1);
       mbar_init(&sh->empty[s], kPassConsumerWarps);
     }
-    sh->abort = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
   }
   // Barriers completed by earlier launches: the counter is a multiple of the grid size when a
   // launch starts and stays below the next multiple until every CTA, this one included, has
   // arrived at the launch's first barrier.
-  if (tid == 32) sh->bar_base = ld_relaxed(&pp.sync->bar_count) / gridDim.x;
+  if (tid == 32) {
+    sh->bar_base = ld_relaxed(&pp.sync->bar_count) / gridDim.x;
+    sh->bar_extra = ld_relaxed(&pp.sync->bar_extra);
+    // an earlier launch gave up a wait and the host has not cleared it yet: this launch's inputs
+    // are not to be trusted, so it does nothing at all
+    sh->abort = *reinterpret_cast<volatile int*>(&pp.sync->error) != 0 ? 1 : 0;
+  }
   if (tid < kPassMaxRows) {  // where the rows sit does not change during the pass
     sh->row_pos[tid] = tid < pp.M ? pp.row_pos[tid] : -1;
     sh->row_seq[tid] = tid < pp.M ? pp.row_seq[tid] : 0;
   }
   __syncthreads();
+  if (sh->abort) return;  // uniform over the CTA: nothing is in flight yet
 
   if (tid >= kPassConsumerThreads) {
     asm volatile("setmaxnreg.dec.sync.aligned.u32 %0;" ::"n"(kPassProducerRegs));

@@ -151,7 +151,8 @@ sample_draft_kernel(const float* logits, int vocab, PassDesc pd, const GenState*
 // are the target's for the token after row i.
 __global__ void __launch_bounds__(kSampleThreads)
 accept_sampled_kernel(GenState* gs_, const float* logits, int vocab, const int* draft_tok, const float* qprob,
-                      const double* qsum, int* seq_tok, int max_seq, int* out_tok, RoundStat* stats) {
+                      const double* qsum, int* seq_tok, int max_seq, int* out_tok, RoundStat* stats,
+                      const int* pass_error) {
   volatile GenState* gs = gs_;
   __shared__ float s_red[kSampleThreads / 32];
   __shared__ double s_scan[kSampleThreads + 33];
@@ -207,6 +208,7 @@ accept_sampled_kernel(GenState* gs_, const float* logits, int vocab, const int* 
     for (int b = 0; b < B; ++b) all &= gs->done[b];
     gs->round += 1;
     gs->all_done = all;
+    gs->pass_error = pass_error ? ld_act(pass_error) : 0;
   }
 }
 

@@ -98,14 +98,25 @@ def _normal(shape, seed: int, device: str) -> torch.Tensor:
     return torch.randn(shape, generator=g, device=device, dtype=torch.float32) * 0.02
 
 
+def _gain(d: int, seed: int, device: str, random_gains: bool) -> torch.Tensor:
+    """RMSNorm gain: ones (the recipe), or uniform in [0.5, 1.5) for tests of the gain path."""
+    if not random_gains:
+        return torch.ones(d, device=device, dtype=torch.float32)
+    g = torch.Generator(device=device)
+    g.manual_seed(seed)
+    return torch.rand(d, generator=g, device=device, dtype=torch.float32) + 0.5
+
+
 def make_weights(shape: ModelShape, skip: Sequence[int], seed: int = MASTER_SEED,
-                 down_scale: float = 0.05, device: str = "cpu") -> Dict:
+                 down_scale: float = 0.05, device: str = "cpu", random_gains: bool = False) -> Dict:
     """Random-init weights as a dict of torch tensors on `device`.
 
     Matrices are [out_features, in_features] row-major.  The draw happens on
     `device` (a CUDA generator and a CPU generator give different numbers for
     the same seed, so a test that needs the same model on both sides draws once
-    and copies).  Storage dtype follows shape.dtype.
+    and copies).  Storage dtype follows shape.dtype.  random_gains=True replaces the
+    unit RMSNorm gains by seeded draws from [0.5, 1.5) (rounded to the storage type), so
+    that a test can see whether every gain reaches the right column.
     """
     st = torch.float32 if shape.dtype == "f32" else torch.bfloat16
     d, f, v = shape.d_model, shape.d_ffn, shape.vocab
@@ -113,7 +124,7 @@ def make_weights(shape: ModelShape, skip: Sequence[int], seed: int = MASTER_SEED
     w: Dict = {"layers": []}
     w["tok_embed"] = _normal((v, d), seed * 1000 + 1, device).to(st)
     w["lm_head"] = _normal((v, d), seed * 1000 + 2, device).to(st)
-    w["final_norm"] = torch.ones(d, device=device, dtype=st)
+    w["final_norm"] = _gain(d, seed * 1000 + 3, device, random_gains).to(st)
     dims = {"wq": (d, d), "wk": (d, d), "wv": (d, d), "wo": (d, d),
             "w_gate": (f, d), "w_up": (f, d), "w_down": (d, f)}
     for l in range(shape.n_layers):
@@ -123,8 +134,8 @@ def make_weights(shape: ModelShape, skip: Sequence[int], seed: int = MASTER_SEED
             if l in skip and name in ("wo", "w_down"):
                 t = t * down_scale
             lw[name] = t.to(st)
-        lw["attn_norm"] = torch.ones(d, device=device, dtype=st)
-        lw["ffn_norm"] = torch.ones(d, device=device, dtype=st)
+        lw["attn_norm"] = _gain(d, seed * 1000 + 10 + l * 16 + 8, device, random_gains).to(st)
+        lw["ffn_norm"] = _gain(d, seed * 1000 + 10 + l * 16 + 9, device, random_gains).to(st)
         w["layers"].append(lw)
     return w
 

@@ -10,10 +10,11 @@ import synth_inputs as si
 from oracle import sdfp_oracle as orc
 
 
-def make_pair(shape, skip, max_seq=160, max_batch=1, k_max=8, flags=0, eos_id=-1, draw_device="cpu"):
+def make_pair(shape, skip, max_seq=160, max_batch=1, k_max=8, flags=0, eos_id=-1, draw_device="cpu",
+              random_gains=False):
     """(library context, oracle Model, weights) on the same weights."""
     pkg.build_library()
-    w = si.make_weights(shape, skip, device=draw_device)
+    w = si.make_weights(shape, skip, device=draw_device, random_gains=random_gains)
     w_gpu = si.weights_to(w, "cuda:0")
     w_cpu = si.weights_to(w, "cpu")
     eng = pkg.Sdfp(shape, w_gpu, max_seq=max_seq, max_batch=max_batch, k_max=k_max, flags=flags, eos_id=eos_id)

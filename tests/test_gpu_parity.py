@@ -385,3 +385,144 @@ def test_fma_and_tensor_paths_agree_closely():
     b = e2.sdfp_forward_logits(toks, 0)
     e2.close()
     assert rel_l2(a, b) < 2e-3
+
+
+# ---- RMSNorm gains other than one ------------------------------------------------------------------
+
+@pytest.mark.parametrize("shape,draw,tol,flags", [
+    (si.TINY, "cpu", 1e-4, 0),
+    (si.TINY_BF16, "cpu", 1e-2, 0),
+    (si.TINY_BF16, "cpu", 1e-2, pkg.FLAG_NO_PASS_KERNEL),
+    (si.TINY_BF16, "cpu", 1e-2, pkg.FLAG_FMA_GEMM),
+    (si.LLAMA7B_4L, "cuda:0", 1e-2, 0),
+    (si.LLAMA7B_4L, "cuda:0", 1e-2, pkg.FLAG_NO_PASS_KERNEL),
+])
+def test_logits_with_random_gains(shape, draw, tol, flags):
+    """Every RMSNorm gain (attention norm, FFN norm, final norm of every layer) drawn from
+    [0.5, 1.5): a gain applied to the wrong column, or not at all, moves the logits by tens of
+    per cent.  Whole-pass kernel, per-operation tensor path and CUDA-core path."""
+    eng, m, _ = make_pair(shape, (1, 2), max_seq=128, flags=flags, draw_device=draw, random_gains=True)
+    try:
+        toks = si.make_prompts(shape.vocab, 1, 45, seed=23)[0].tolist()
+        got, ref = _logits_both(eng, m, toks, [17, 1, 5, 22])
+        assert rel_l2(got, ref) < tol
+        assert max(rel_l2(got[r], ref[r]) for r in range(45)) < tol
+        got, ref = _logits_both(eng, m, toks, [33, 12], layers=[0, 3])
+        assert rel_l2(got, ref) < tol
+        # and the gains matter: the same tokens through unit gains are far away
+        plain = orc.Model.from_shape(shape, si.make_weights(shape, (1, 2), device="cpu"))
+        if draw == "cpu":
+            far = orc.CachedLM(plain, max_seq=64).feed(toks[:8], 0).numpy()
+            assert rel_l2(got[:8], far) > 0.05
+    finally:
+        eng.close()
+
+
+# ---- one arithmetic path per context: wide contexts (batch x (k+1) > 16 rows) ----------------------
+
+@pytest.mark.parametrize("batch,k", [(4, 4), (4, 8), (8, 2), (8, 4), (8, 8)])
+def test_wide_batches_bf16(batch, k):
+    """bf16 contexts whose verify pass exceeds the whole-pass kernel's 16 rows (20 .. 72 rows here)
+    run every pass on the per-operation kernels.  Speculative output equals autoregressive
+    output bit for bit, every sequence equals its solo run in the same context (tokens and
+    acceptance counts: ragged across the batch), and every stream passes the oracle."""
+    eng, m, _ = make_pair(si.TINY_BF16, (1, 2), max_seq=160, max_batch=batch, k_max=k)
+    try:
+        prompts = si.make_prompts(m.vocab, batch, 24, seed=50 + batch)
+        n_new = 36
+        out = eng.sdfp_generate(prompts, k, n_new)
+        ar = eng.sdfp_generate(prompts, 0, n_new)
+        assert out.tokens == ar.tokens
+        ragged = set()
+        for b in range(batch):
+            solo = eng.sdfp_generate(prompts[b:b + 1], k, n_new)
+            assert solo.tokens[0] == out.tokens[b]
+            acc_b = [int(a) for a, d in zip(out.stats[:, b, 1], out.stats[:, b, 0]) if d > 0]
+            assert acc_b == solo.stats[:, 0, 1].tolist()
+            ragged.add(tuple(acc_b))
+            check_stream_against_oracle(m, prompts[b].tolist(), out.tokens[b])
+        assert len(ragged) > 1                      # the sequences really accept differently
+        assert int(out.stats[:, :, 2].sum()) == batch * n_new
+    finally:
+        eng.close()
+
+
+def test_wide_batch_7b_shape():
+    """Batch 8, k = 8 (72-row verify passes, 16-row first draft passes) at the 7B layer shapes."""
+    shape = si.LLAMA7B_4L
+    eng, m, _ = make_pair(shape, (1, 2), max_seq=128, max_batch=8, k_max=8, draw_device="cuda:0")
+    try:
+        prompts = si.make_prompts(shape.vocab, 8, 40, seed=60)
+        out = eng.sdfp_generate(prompts, 8, 20)
+        ar = eng.sdfp_generate(prompts, 0, 20)
+        assert out.tokens == ar.tokens
+        for b in (0, 3, 7):
+            solo = eng.sdfp_generate(prompts[b:b + 1], 8, 20)
+            assert solo.tokens[0] == out.tokens[b]
+            check_stream_against_oracle(m, prompts[b].tolist(), out.tokens[b])
+        # rows of one forward call: the same bits whether fed one by one or 72 at a time
+        toks = si.make_prompts(shape.vocab, 1, 72, seed=61)[0].tolist()
+        blk = eng.sdfp_forward_logits(toks, 0)
+        one = np.concatenate([eng.sdfp_forward_logits(toks[i:i + 1], i) for i in range(72)])
+        assert np.array_equal(one.view(np.uint32), blk.view(np.uint32))
+        ref = orc.CachedLM(m, max_seq=128).feed(toks, 0).numpy()
+        assert max(rel_l2(blk[r], ref[r]) for r in range(72)) < 1e-2
+    finally:
+        eng.close()
+
+
+def test_create_accepts_72_rows_and_rejects_more():
+    w = si.weights_to(si.make_weights(si.TINY_BF16, (1, 2)), "cuda:0")
+    with pytest.raises(pkg.SdfpError):
+        pkg.Sdfp(si.TINY_BF16, w, max_seq=64, max_batch=9, k_max=8)       # 81 rows
+    eng = pkg.Sdfp(si.TINY_BF16, w, max_seq=64, max_batch=8, k_max=9)     # 80 rows
+    eng.close()
+
+
+# ---- the slot hand-back of the whole-pass kernel, many times over ---------------------------------
+
+def test_pass_kernel_soak_16_rows(l7b4):
+    """2000 16-row passes over the same tokens and positions: every one must give, bit for bit,
+    the logits of 16 single-row passes.  (A weight slot handed back before its tile reads had
+    completed once corrupted about one pass in 200 at full speed, only in wide passes.)"""
+    eng, m = l7b4
+    toks = si.make_prompts(m.vocab, 1, 16, seed=24)[0].tolist()
+    one = np.concatenate([eng.sdfp_forward_logits(toks[i:i + 1], i) for i in range(16)]).view(np.uint32)
+    bad = 0
+    for it in range(2000):
+        blk = eng.sdfp_forward_logits(toks, 0).view(np.uint32)
+        bad += int(not np.array_equal(blk, one))
+    assert bad == 0
+
+
+# ---- a bounded wait that runs out --------------------------------------------------------------------
+
+def test_wait_that_runs_out_returns_timeout(tiny_bf16):
+    """Failure path of the whole-pass kernel's waits, without faulting anything: the next pass is
+    told to expect one barrier arrival more than the grid has, with a 20 ms limit.  The call
+    must come back quickly with SDFP_ETIMEOUT and the name of the wait, and the context must
+    work again afterwards (same tokens as before)."""
+    import time
+    eng, m = tiny_bf16
+    prompt = si.make_prompts(m.vocab, 1, 16)
+    before = eng.sdfp_generate(prompt, 4, 24)
+    toks = prompt[0].tolist()
+    logits_before = eng.sdfp_forward_logits(toks, 0)
+    eng.sdfp_debug_expire_next_wait(20_000_000)
+    t0 = time.perf_counter()
+    with pytest.raises(pkg.SdfpError) as ei:
+        eng.sdfp_forward_logits(toks, 0)
+    assert time.perf_counter() - t0 < 1.0
+    assert ei.value.code == -5 and "grid barrier" in str(ei.value)
+    assert np.array_equal(eng.sdfp_forward_logits(toks, 0).view(np.uint32), logits_before.view(np.uint32))
+    # the same inside a generate call: the round loop stops at the first round
+    eng.sdfp_debug_expire_next_wait(20_000_000)
+    t0 = time.perf_counter()
+    with pytest.raises(pkg.SdfpError) as ei:
+        eng.sdfp_generate(prompt, 4, 24)
+    assert time.perf_counter() - t0 < 1.5
+    assert ei.value.code == -5
+    after = eng.sdfp_generate(prompt, 4, 24)
+    assert after.tokens == before.tokens and np.array_equal(after.stats, before.stats)
+    ar = eng.sdfp_generate(prompt, 0, 24)
+    assert ar.tokens == before.tokens

@@ -88,3 +88,57 @@ def test_sampling_draft_equal_target_accepts_all(tiny64):
     finally:
         eng.sdfp_set_draft_layers(si.keep_mask(4, (1, 2)))
     assert (out.stats[:, 0, 1] == 4).all()
+
+
+# ---- vocabularies where a thread of the draw owns several elements ---------------------------------
+
+def test_sampled_tokens_match_oracle_vocab_2048():
+    """Vocabulary 2048 with 1024 threads: every thread sums a two-element segment, the scan runs
+    over non-trivial totals and the owner walks its segment.  Same rule as at vocabulary 64."""
+    eng, m, _ = make_pair(si.TINY, (1, 2), max_seq=64, k_max=6)
+    try:
+        prompt = si.make_prompts(m.vocab, 1, 16)
+        T = 1.0 / 8.0
+        same = total = 0
+        for seed in range(40):
+            out = eng.sdfp_generate(prompt, 4, 24, temperature=T, seed=seed)
+            ref = orc.spec_generate(orc.CachedLM(m, max_seq=64), orc.CachedLM(m, [0, 3], max_seq=64),
+                                    prompt[0].tolist(), 4, 24, temperature=T, seed=seed)
+            total += 1
+            if out.tokens[0] == ref.tokens:
+                same += 1
+                assert out.stats[:, 0, 1].tolist() == [r.accepted for r in ref.rounds]
+            ar = eng.sdfp_generate(prompt, 0, 24, temperature=T, seed=seed)
+            ar_ref = orc.ar_generate(orc.CachedLM(m, max_seq=64), prompt[0].tolist(), 24, temperature=T, seed=seed)
+            total += 1
+            same += (ar.tokens[0] == ar_ref.tokens)
+        assert same >= total - 2
+    finally:
+        eng.close()
+
+
+def test_sampled_tokens_match_oracle_vocab_32000():
+    """The sampled configuration's real vocabulary and draft length (V = 32000, k = 6, temperature
+    1) on the 7B layer shapes: 32-element segments per thread.  Tokens and acceptance counts
+    against the oracle's loop, seed by seed."""
+    shape = si.LLAMA7B_4L
+    eng, m, _ = make_pair(shape, (1, 2), max_seq=64, k_max=6, draw_device="cuda:0")
+    try:
+        prompt = si.make_prompts(shape.vocab, 1, 12, seed=31)
+        same = total = 0
+        accepted = drafted = 0
+        for seed in range(6):
+            out = eng.sdfp_generate(prompt, 6, 14, temperature=1.0, seed=seed)
+            ref = orc.spec_generate(orc.CachedLM(m, max_seq=64), orc.CachedLM(m, [0, 3], max_seq=64),
+                                    prompt[0].tolist(), 6, 14, temperature=1.0, seed=seed)
+            total += 1
+            accepted += int(out.stats[:, 0, 1].sum())
+            drafted += int(out.stats[:, 0, 0].sum())
+            if out.tokens[0] == ref.tokens:
+                same += 1
+                assert out.stats[:, 0, 1].tolist() == [r.accepted for r in ref.rounds]
+                assert out.stats[:, 0, 2].tolist() == [r.committed for r in ref.rounds]
+        assert same >= total - 1
+        assert 0 < accepted < drafted                  # both outcomes of the accept test occurred
+    finally:
+        eng.close()

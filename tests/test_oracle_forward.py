@@ -185,6 +185,71 @@ def test_two_token_attention_worked_by_hand():
     assert r1[0].tolist() == pytest.approx(exp_rows[1], rel=1e-12)
 
 
+def test_two_heads_partition_contiguous_blocks_worked_by_hand():
+    """d=4, two heads of width 2, wq=wk=wv=wo=I, T=2: head h owns dimensions 2h, 2h+1 of q, k
+    and v (contiguous blocks, the LLaMA layout), each head has its own softmax over the two
+    keys, and the two heads get different attention weights.  Everything is worked in scalars;
+    a layout that interleaved the heads (dimensions h, h+2) pairs different numbers in the
+    rotation and in the dot products and gives other values."""
+    m = _hand_model(4, 2, 2, 2, 4)
+    e0, e1 = [1.0, 2.0, -1.0, 0.5], [-0.5, 1.5, 2.0, 1.0]
+    m.w["tok_embed"][0] = torch.tensor(e0, dtype=torch.float64)
+    m.w["tok_embed"][1] = torch.tensor(e1, dtype=torch.float64)
+    lw = m.w["layers"][0]
+    for name in ("wq", "wk", "wv", "wo"):
+        for i in range(4):
+            lw[name][i, i] = 1.0
+    for i in range(4):
+        m.w["lm_head"][i, i] = 1.0
+
+    def norm(v):
+        r = math.sqrt(sum(x * x for x in v) / 4 + 1e-5)
+        return [x / r for x in v]
+
+    def rot(a, b, pos):                   # head_dim 2: one pair per head, frequency 1
+        c, s = math.cos(pos), math.sin(pos)
+        return [a * c - b * s, b * c + a * s]
+
+    x0, x1 = norm(e0), norm(e1)
+    a1, probs = [], []
+    for h in range(2):
+        lo, hi = 2 * h, 2 * h + 1
+        k0 = rot(x0[lo], x0[hi], 0)
+        k1 = rot(x1[lo], x1[hi], 1)
+        q1 = k1                           # wq = wk
+        s10 = (q1[0] * k0[0] + q1[1] * k0[1]) / math.sqrt(2)
+        s11 = (q1[0] * k1[0] + q1[1] * k1[1]) / math.sqrt(2)
+        mx = max(s10, s11)
+        w0, w1 = math.exp(s10 - mx), math.exp(s11 - mx)
+        p0, p1 = w0 / (w0 + w1), w1 / (w0 + w1)
+        probs.append(p0)
+        a1 += [p0 * x0[lo] + p1 * x1[lo], p0 * x0[hi] + p1 * x1[hi]]      # v = x̂, not rotated
+    assert abs(probs[0] - probs[1]) > 0.02                                # the heads really differ
+    h_row0 = [e0[i] + x0[i] for i in range(4)]                            # row 0 sees only itself
+    h_row1 = [e1[i] + a1[i] for i in range(4)]
+    expect = [norm(h_row0), norm(h_row1)]                                 # FFN is zero
+    got = o.forward_nocache(m, [0, 1])
+    assert got[0].tolist() == pytest.approx(expect[0], rel=1e-12)
+    assert got[1].tolist() == pytest.approx(expect[1], rel=1e-12)
+    lm = o.CachedLM(m, max_seq=4)
+    r0 = lm.feed([0], 0)
+    r1 = lm.feed([1], 1)
+    assert r0[0].tolist() == pytest.approx(expect[0], rel=1e-12)
+    assert r1[0].tolist() == pytest.approx(expect[1], rel=1e-12)
+    both = o.CachedLM(m, max_seq=4).feed([0, 1], 0)
+    assert both[1].tolist() == pytest.approx(expect[1], rel=1e-12)
+    # the interleaved reading (head h = dimensions h, h+2) worked the same way gives other numbers
+    alt = []
+    for h in range(2):
+        lo, hi = h, h + 2
+        k0, k1 = rot(x0[lo], x0[hi], 0), rot(x1[lo], x1[hi], 1)
+        s10 = (k1[0] * k0[0] + k1[1] * k0[1]) / math.sqrt(2)
+        s11 = (k1[0] * k1[0] + k1[1] * k1[1]) / math.sqrt(2)
+        w0, w1 = math.exp(s10 - max(s10, s11)), math.exp(s11 - max(s10, s11))
+        alt.append(w0 / (w0 + w1))
+    assert abs(alt[0] - probs[0]) > 1e-3 or abs(alt[1] - probs[1]) > 1e-3
+
+
 def test_uniform_attention_is_causal_running_mean():
     """wq = 0 makes every score 0, so attention is the running mean of v (textbook special case)."""
     shape = si.ModelShape("t", 1, 32, 2, 16, 48, 40)

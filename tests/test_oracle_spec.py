@@ -195,6 +195,21 @@ def test_losslessness_identity_on_real_distributions(tiny64):
     assert torch.equal(o.residual_distribution(p, p), p)
 
 
+def test_softmax_temperature_literals():
+    """The temperature DIVIDES the logits (reading R4; p and q of Eq. 2 are softmax(logits / T)).
+    With logits (0, ln 2): T = 1 gives (1/3, 2/3); T = 1/2 doubles the gap, (1/5, 4/5); T = 2
+    halves it, (1, sqrt 2) / (1 + sqrt 2).  Multiplying by T instead would swap the last two."""
+    lg = torch.tensor([0.0, math.log(2.0)], dtype=torch.float32)
+    assert o.softmax_T(lg, 1.0).tolist() == pytest.approx([1 / 3, 2 / 3], rel=1e-6)
+    assert o.softmax_T(lg, 0.5).tolist() == pytest.approx([1 / 5, 4 / 5], rel=1e-6)
+    r2 = math.sqrt(2.0)
+    assert o.softmax_T(lg, 2.0).tolist() == pytest.approx([1 / (1 + r2), r2 / (1 + r2)], rel=1e-6)
+    # three logits, shifted by a constant: the shift cancels, the result stays normalised
+    p = o.softmax_T(torch.tensor([100.0, 100.0 + math.log(3.0), 100.0 - math.log(2.0)]), 1.0)
+    assert p.tolist() == pytest.approx([1 / 4.5, 3 / 4.5, 0.5 / 4.5], rel=1e-5)
+    assert float(p.sum()) == pytest.approx(1.0, abs=1e-12)
+
+
 def test_categorical_inverse_cdf():
     w = torch.tensor([0.0, 2.0, 0.0, 1.0, 1.0])          # cdf: 0, .5, .5, .75, 1
     assert o.categorical(w, 0.01) == 1

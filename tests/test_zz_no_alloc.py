@@ -64,3 +64,36 @@ def test_static_scratch_rejects_what_does_not_fit():
         assert np.array_equal(ok.view(np.uint32), eng.sdfp_forward_logits(toks[:5], 0).view(np.uint32))
     finally:
         eng.close()
+
+
+def test_static_call_allocates_nothing_and_leaves_the_context_intact():
+    """The promise itself: once the first call on the device has looked the array up, a static call
+    leaves the device's free memory exactly where it was (no cudaMalloc, no pool growth), a refused
+    call likewise, and afterwards the context still generates what a fresh context generates (the
+    static call borrows the context's scratch pointers and must hand them back, also on the error
+    return)."""
+    import torch
+    shape = si.LLAMA7B_4L
+    kw = dict(max_seq=2200, flags=pkg.FLAG_NO_PASS_KERNEL, draw_device="cuda:0")
+    eng, m, _ = make_pair(shape, (1, 2), **kw)
+    fresh, _, _ = make_pair(shape, (1, 2), **kw)
+    try:
+        toks = si.make_prompts(shape.vocab, 1, 70, seed=25)[0].tolist()
+        eng.sdfp_forward_logits_static(toks[:8], 0)              # resolves the symbol on this device
+        torch.cuda.synchronize()
+        free0, _ = torch.cuda.mem_get_info()
+        for start, n in ((0, 40), (40, 30), (0, 1)):
+            eng.sdfp_forward_logits_static(toks[start:start + n], start)
+        with pytest.raises(pkg.SdfpError):                        # 64 rows at a context of 2164 tokens: refused
+            eng.sdfp_forward_logits_static(toks[:64], 2100)
+        torch.cuda.synchronize()
+        free1, _ = torch.cuda.mem_get_info()
+        assert free1 == free0
+        prompt = si.make_prompts(shape.vocab, 1, 90, seed=26)     # context beyond one 64-key chunk
+        for k in (4, 0):
+            a = eng.sdfp_generate(prompt, k, 20)
+            b = fresh.sdfp_generate(prompt, k, 20)
+            assert a.tokens == b.tokens and np.array_equal(a.stats, b.stats)
+    finally:
+        eng.close()
+        fresh.close()
