@@ -61,6 +61,9 @@ typedef enum { SDFP_F32 = 0, SDFP_BF16 = 1 } sdfp_dtype;
 #define SDFP_FLAG_FMA_GEMM 4u /* bf16 models: CUDA-core FMA GEMM instead of the tensor path  */
 #define SDFP_FLAG_NO_PASS_KERNEL 8u /* bf16 models: one kernel per operation instead of the
                                        persistent whole-pass kernel                            */
+#define SDFP_FLAG_NO_DENSE 16u      /* bf16 models: no tcgen05 path (the prompt goes through the
+                                       decode kernels in chunks; contexts too wide for the
+                                       whole-pass kernel run mma.sync kernels per operation)  */
 
 /*
  * Model and capacity description.  The decoder is the LLaMA-2 architecture the

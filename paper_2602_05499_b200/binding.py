@@ -13,7 +13,7 @@ import numpy as np
 from .build import LIB_PATH
 
 SDFP_F32, SDFP_BF16 = 0, 1
-FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_FMA_GEMM, FLAG_NO_PASS_KERNEL = 1, 2, 4, 8
+FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_FMA_GEMM, FLAG_NO_PASS_KERNEL, FLAG_NO_DENSE = 1, 2, 4, 8, 16
 
 EXPORTS = ["sdfp_create", "sdfp_set_draft_layers", "sdfp_generate", "sdfp_forward_logits",
            "sdfp_forward_logits_static", "sdfp_get_timing", "sdfp_time_linear", "sdfp_time_pass",

@@ -27,7 +27,9 @@
 #include "linear_mma.cuh"
 #include "misc_kernels.cuh"
 #include "pass_kernel.cuh"
+#include "prefill_attention.cuh"
 #include "sampling.cuh"
+#include "umma_linear.cuh"
 
 using namespace sdfp;
 
@@ -40,6 +42,8 @@ struct LayerWeights {
   void* wo = nullptr;    // packed [d, d]
   void* gu = nullptr;    // packed [2f, d]
   void* down = nullptr;  // packed [d, f]
+  // the same matrices as tcgen05 operand images (dense path), null when that path is off
+  void *um_qkv = nullptr, *um_wo = nullptr, *um_gu = nullptr, *um_down = nullptr;
   float* attn_gain = nullptr;
   float* ffn_gain = nullptr;
 };
@@ -69,6 +73,7 @@ struct sdfp_ctx {
 
   // activations / scratch
   float *h = nullptr, *q = nullptr, *att = nullptr, *u = nullptr, *logits = nullptr;
+  float* h_fork = nullptr;  // dense prompt pass: the residual rows where the draft leaves the target
   float *part_o = nullptr, *part_ml = nullptr;
   int* attn_counters = nullptr;
   int n_chunks_cap = 0;
@@ -101,6 +106,16 @@ struct sdfp_ctx {
   int pass_slots[3] = {0, 0, 0};  // ring slots of the instantiation with 1 and with 2 column groups
   size_t pass_smem = 0;
   int pass_grid = 0;
+  // dense path on tcgen05 (bf16 tensor path): the prompt pass of every context, and every pass of
+  // a context whose widest pass does not fit the whole-pass kernel
+  bool use_dense = false;
+  bool dense_decode = false;       // ... this context's decode passes run on it as well
+  void* um_lm_head = nullptr;
+  unsigned char* um_x = nullptr;   // activation image, rows_cap (rounded to 128) x widest K
+  float* um_partial = nullptr;
+  int *um_flags = nullptr, *um_error = nullptr;
+  int rows_cap = kMaxRows;         // rows the activation buffers h, q, att, u and the row plan hold
+  int max_smem_optin = 0;
   bool own_stream = false;
   sdfp_timing timing{};
   cudaEvent_t ev[3] = {nullptr, nullptr, nullptr};
@@ -173,7 +188,38 @@ int linear_grid_fma(const sdfp_ctx* c, int n_pairs) {
   return std::max(1, std::min(want, c->num_sms * 8));
 }
 
+// Linear layer on the tcgen05 path: activation image (RMSNorm folded in), then the stream-K kernel.
+// Launched in plain stream order (no programmatic dependent launch): the kernel holds all of an
+// SM's tensor memory and nearly all of its shared memory, so nothing should share the SM with it.
+cudaError_t run_dense_linear(sdfp_ctx* c, const void* w_img, const float* x, int ldx, int rows, int K, int n_pairs,
+                             const float* gain, const EpiParams& ep) {
+  const int RB = rows >= kUmMaxRB ? kUmMaxRB : ((rows + 15) / 16) * 16;
+  const int KB = (K + kUmBK - 1) / kUmBK;
+  cudaError_t e = launch(c, prep_rows_kernel, dim3((rows + 7) / 8), dim3(kPrepThreads), 0, x, ldx, rows, K, gain, c->cfg.rms_eps,
+                         c->um_x, RB, KB);
+  if (e != cudaSuccess) return e;
+  UmmaParams p{};
+  p.W = reinterpret_cast<const unsigned char*>(w_img);
+  p.X = c->um_x;
+  p.n_ft = (n_pairs + 63) / 64;
+  p.n_rb = (rows + RB - 1) / RB;
+  p.KB = KB;
+  p.RB = RB;
+  p.M = rows;
+  p.n_pairs = n_pairs;
+  p.n_stages = umma_stages_for(RB, c->max_smem_optin);
+  p.partial = c->um_partial;
+  p.flags = c->um_flags;
+  p.error = c->um_error;
+  p.ep = ep;
+  c->launches += 1;
+  umma_linear_kernel<<<c->num_sms, kUmThreads, umma_smem_bytes(RB, p.n_stages), c->stream>>>(p);
+  return cudaGetLastError();
+}
+
 cudaError_t run_linear(sdfp_ctx* c, const LinearCall& lc) {
+  if (c->dense_decode)
+    return run_dense_linear(c, lc.w, lc.x, lc.ldx, lc.rows, lc.K, lc.n_pairs, lc.gain, lc.ep);
   if (c->use_mma)
     return launch_linear_mma(c->L, c->num_sms, lc.w, lc.x, lc.ldx, lc.rows, lc.K, lc.n_pairs, lc.gain, c->cfg.rms_eps, lc.ep);
   const dim3 grid(linear_grid_fma(c, lc.n_pairs)), block(kFmaThreads);
@@ -410,6 +456,9 @@ cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool w
 
 // ---- one forward pass ------------------------------------------------------------------
 
+// prompts shorter than this go through the decode kernels in chunks (a handful of launches)
+constexpr int kDenseMinRows = 16;
+
 enum Decide { DECIDE_NONE = 0, DECIDE_LOGITS = 1, DECIDE_ARGMAX = 2, DECIDE_SAMPLE_DRAFT = 3 };
 
 // rows: total rows; rows_per_seq for the attention grouping; n_chunks bounds the context.
@@ -498,8 +547,29 @@ int enqueue_round(sdfp_ctx* c, int k, int batch, bool sampled, int n_chunks) {
 
 // ---- weights ------------------------------------------------------------------------------
 
+// the tcgen05 operand image of a matrix (see umma_linear.cuh)
+int pack_dense_image(sdfp_ctx* c, void** dst, PackSrc ps, int n_pairs, int K) {
+  const int n_ft = (n_pairs + 63) / 64, KB = (K + kUmBK - 1) / kUmBK;
+  __nv_bfloat16* p = nullptr;
+  if (int r = dev_alloc(c, &p, (size_t)n_ft * KB * (kUmABytes / 2))) return r;
+  pack_umma_kernel<<<1184, 256, 0, c->stream>>>(p, ps, n_pairs, K, n_ft, KB);
+  CU_OK(c, cudaGetLastError());
+  *dst = p;
+  return 0;
+}
+
+// A matrix in the layout(s) this context's kernels read: `dst` for the whole-pass / per-operation
+// kernels, `img` (may be null) for the dense path.  A context whose decode passes run on the dense
+// path reads only images: `dst` then points to the image as well.
 template <typename WT>
-int pack_matrix(sdfp_ctx* c, void** dst, PackSrc ps, int n_pairs, int K) {
+int pack_matrix(sdfp_ctx* c, void** dst, void** img, PackSrc ps, int n_pairs, int K) {
+  if (c->use_dense && img) {
+    if (int r = pack_dense_image(c, img, ps, n_pairs, K)) return r;
+    if (c->dense_decode) {
+      *dst = *img;
+      return 0;
+    }
+  }
   const int n_groups = (n_pairs / 8 + kUnitTiles - 1) / kUnitTiles;
   const size_t n = c->use_mma ? (size_t)n_groups * (K / 16) * (kUnitBytes / 2) : (size_t)n_pairs * 2 * K;
   WT* p = nullptr;
@@ -532,14 +602,17 @@ int load_weights(sdfp_ctx* c, const sdfp_weights* w) {
     if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] || !w->w_down[l] ||
         !w->attn_norm[l] || !w->ffn_norm[l])
       return fail(c, SDFP_EINVAL, "layer %d has a NULL weight pointer", l);
-    if (int r = pack_matrix<WT>(c, &lw.qkv, PackSrc{w->wq[l], w->wk[l], w->wv[l], 0, H, hd}, 3 * d / 2, d)) return r;
-    if (int r = pack_matrix<WT>(c, &lw.wo, PackSrc{w->wo[l], nullptr, nullptr, 2, H, hd}, d / 2, d)) return r;
-    if (int r = pack_matrix<WT>(c, &lw.gu, PackSrc{w->w_gate[l], w->w_up[l], nullptr, 1, H, hd}, f, d)) return r;
-    if (int r = pack_matrix<WT>(c, &lw.down, PackSrc{w->w_down[l], nullptr, nullptr, 2, H, hd}, d / 2, f)) return r;
+    if (int r = pack_matrix<WT>(c, &lw.qkv, &lw.um_qkv, PackSrc{w->wq[l], w->wk[l], w->wv[l], 0, H, hd}, 3 * d / 2, d)) return r;
+    if (int r = pack_matrix<WT>(c, &lw.wo, &lw.um_wo, PackSrc{w->wo[l], nullptr, nullptr, 2, H, hd}, d / 2, d)) return r;
+    if (int r = pack_matrix<WT>(c, &lw.gu, &lw.um_gu, PackSrc{w->w_gate[l], w->w_up[l], nullptr, 1, H, hd}, f, d)) return r;
+    if (int r = pack_matrix<WT>(c, &lw.down, &lw.um_down, PackSrc{w->w_down[l], nullptr, nullptr, 2, H, hd}, d / 2, f)) return r;
     if (int r = widen_gain<WT>(c, &lw.attn_gain, w->attn_norm[l], d)) return r;
     if (int r = widen_gain<WT>(c, &lw.ffn_gain, w->ffn_norm[l], d)) return r;
   }
-  if (int r = pack_matrix<WT>(c, &c->lm_head, PackSrc{w->lm_head, nullptr, nullptr, 2, H, hd}, g.vocab / 2, d)) return r;
+  // the prompt pass needs no logits: only contexts that decode on the dense path get an lm-head image
+  if (int r = pack_matrix<WT>(c, &c->lm_head, c->dense_decode ? &c->um_lm_head : nullptr,
+                              PackSrc{w->lm_head, nullptr, nullptr, 2, H, hd}, g.vocab / 2, d))
+    return r;
   if (int r = widen_gain<WT>(c, &c->final_gain, w->final_norm, d)) return r;
   WT* e = nullptr;
   if (int r = dev_alloc(c, &e, (size_t)g.vocab * d)) return r;
@@ -668,9 +741,23 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   const int widest = g.max_batch * std::max(g.k_max + 1, 2);
   c->use_pass = c->use_mma && !(g.flags & SDFP_FLAG_NO_PASS_KERNEL) && prop.cooperativeLaunch && g.d_model >= 64 &&
                 g.n_heads <= kPassMaxHeads && g.d_model / 128 + 1 <= kSsqMaxGroups && widest <= kPassMaxRows;
+  int optin = 0;
+  cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
+  c->max_smem_optin = optin;
+  c->use_dense = c->use_mma && !(g.flags & SDFP_FLAG_NO_DENSE);
+  c->dense_decode = c->use_dense && !c->use_pass && !(g.flags & SDFP_FLAG_NO_PASS_KERNEL);
+  if (c->use_dense) {
+    c->rows_cap = std::max((int)kMaxRows, g.max_seq);
+    if (cudaFuncSetAttribute(umma_linear_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, optin) != cudaSuccess ||
+        cudaFuncSetAttribute(prefill_attention_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)prefill_attention_smem<64>()) != cudaSuccess ||
+        cudaFuncSetAttribute(prefill_attention_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)prefill_attention_smem<128>()) != cudaSuccess) {
+      c->err = "dense-path kernel configuration failed";
+      return bail(SDFP_ECUDA);
+    }
+  }
   if (c->use_pass) {
-    int optin = 0;
-    cudaDeviceGetAttribute(&optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
     const cudaError_t pe = g.head_dim == 128 ? configure_pass_t<128>(c, optin) : configure_pass_t<64>(c, optin);
     if (pe != cudaSuccess) {
       c->err = std::string("pass kernel configuration failed: ") + cudaGetErrorString(pe);
@@ -704,25 +791,34 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
       return bail(SDFP_ECUDA);
     }
   }
-  const size_t R = kMaxRows;
+  const size_t R = (size_t)c->rows_cap;  // prompt rows on the dense path, else the rows of the widest decode pass
   c->n_chunks_cap = std::max(2, (g.max_seq + kAttnChunk - 1) / kAttnChunk);  // >= 16 rows x kAttnSplits partials
   c->stats_cap = g.max_seq;
   if ((r = dev_alloc(c, &c->h, R * g.d_model, true)) || (r = dev_alloc(c, &c->q, R * g.d_model, true)) ||
       (r = dev_alloc(c, &c->att, R * g.d_model, true)) || (r = dev_alloc(c, &c->u, R * g.d_ffn, true)) ||
-      (r = dev_alloc(c, &c->logits, R * g.vocab, true)) ||
-      (r = dev_alloc(c, &c->part_o, R * g.n_heads * c->n_chunks_cap * g.head_dim)) ||
-      (r = dev_alloc(c, &c->part_ml, R * g.n_heads * c->n_chunks_cap * 2)) ||
-      (r = dev_alloc(c, &c->attn_counters, R * g.n_heads, true)) || (r = dev_alloc(c, &c->plan.row_pos, R, true)) ||
+      (r = dev_alloc(c, &c->logits, (size_t)kMaxRows * g.vocab, true)) ||
+      (r = dev_alloc(c, &c->part_o, (size_t)kMaxRows * g.n_heads * c->n_chunks_cap * g.head_dim)) ||
+      (r = dev_alloc(c, &c->part_ml, (size_t)kMaxRows * g.n_heads * c->n_chunks_cap * 2)) ||
+      (r = dev_alloc(c, &c->attn_counters, (size_t)kMaxRows * g.n_heads, true)) || (r = dev_alloc(c, &c->plan.row_pos, R, true)) ||
       (r = dev_alloc(c, &c->plan.row_seq, R, true)) || (r = dev_alloc(c, &c->plan.row_tok, R, true)) ||
       (r = dev_alloc(c, &c->seq_tok, (size_t)g.max_batch * g.max_seq, true)) ||
       (r = dev_alloc(c, &c->draft_tok, (size_t)kMaxBatch * kMaxK, true)) ||
       (r = dev_alloc(c, &c->tgt_tok, (size_t)kMaxBatch * (kMaxK + 1), true)) ||
-      (r = dev_alloc(c, &c->row_argmax, R, true)) || (r = dev_alloc(c, &c->out_tok, (size_t)g.max_batch * g.max_seq, true)) ||
-      (r = dev_alloc(c, &c->fwd_tok, R, true)) ||
+      (r = dev_alloc(c, &c->row_argmax, (size_t)kMaxRows, true)) || (r = dev_alloc(c, &c->out_tok, (size_t)g.max_batch * g.max_seq, true)) ||
+      (r = dev_alloc(c, &c->fwd_tok, (size_t)kMaxRows, true)) ||
       (r = dev_alloc(c, &c->qprob, (size_t)g.max_batch * std::max(1, g.k_max) * g.vocab, true)) ||
       (r = dev_alloc(c, &c->qsum, (size_t)kMaxBatch * kMaxK, true)) || (r = dev_alloc(c, &c->gs, 1, true)) ||
       (r = dev_alloc(c, &c->stats, (size_t)c->stats_cap * g.max_batch, true)))
     return bail(r);
+  if (c->use_dense) {
+    const size_t rows128 = ((R + 127) / 128) * 128;
+    const size_t kmax = (size_t)(((std::max(g.d_model, g.d_ffn) + kUmBK - 1) / kUmBK) * kUmBK);
+    if ((r = dev_alloc(c, &c->um_x, rows128 * kmax * 4, true)) ||
+        (r = dev_alloc(c, &c->um_partial, (size_t)c->num_sms * kUmMaxRB * kUmFeat)) ||
+        (r = dev_alloc(c, &c->um_flags, (size_t)c->num_sms, true)) || (r = dev_alloc(c, &c->um_error, 1, true)) ||
+        (r = dev_alloc(c, &c->h_fork, R * g.d_model)))
+      return bail(r);
+  }
   if (c->use_pass) {
     if ((r = dev_alloc(c, &c->psync, 1, true)) ||
         (r = dev_alloc(c, &c->split_partials, (size_t)c->pass_grid * kUnitTiles * 2 * 64, true)) ||
@@ -768,6 +864,21 @@ extern "C" int sdfp_set_draft_layers(sdfp_ctx* c, const uint8_t* keep_mask) {
 
 namespace {
 
+int check_dense_error(sdfp_ctx* c) {
+  if (!c->use_dense) return 0;
+  int e = 0;
+  CU_OK(c, cudaMemcpyAsync(&e, c->um_error, sizeof e, cudaMemcpyDeviceToHost, c->stream));
+  CU_OK(c, cudaStreamSynchronize(c->stream));
+  if (e == 0) return 0;
+  cudaMemsetAsync(c->um_error, 0, sizeof(int), c->stream);
+  cudaMemsetAsync(c->um_flags, 0, (size_t)c->num_sms * sizeof(int), c->stream);
+  cudaStreamSynchronize(c->stream);
+  static const char* const what[] = {"", "pipeline stage never freed", "pipeline stage never filled", "accumulator never freed",
+                                     "accumulator never finished", "partial accumulator of a cut tile never posted"};
+  return fail(c, SDFP_ETIMEOUT, "dense linear kernel gave up a wait (%s); results of this call are invalid",
+              e >= 1 && e <= 5 ? what[e] : "unknown");
+}
+
 // A failed wait inside the pass kernel leaves its code in device memory; turn it into an error
 // and put the synchronisation words back to their initial state.
 int check_pass_error(sdfp_ctx* c) {
@@ -807,6 +918,7 @@ int forward_logits_passes(sdfp_ctx* c, bool draft, const int32_t* tokens, int ro
                              cudaMemcpyDeviceToHost, c->stream));
   }
   CU_OK(c, cudaStreamSynchronize(c->stream));
+  if (int r = check_dense_error(c)) return r;
   return check_pass_error(c);
 }
 
@@ -830,6 +942,87 @@ int prefill_range(sdfp_ctx* c, bool draft, int b, int from, int to) {
     const int n_chunks = (s + cnt + kAttnChunk - 1) / kAttnChunk;
     if (int r = enqueue_pass(c, pd, draft, rows, rps, n_chunks, DECIDE_NONE)) return r;
   }
+  return 0;
+}
+
+// ---- the prompt pass on the dense path ---------------------------------------------------------------
+//
+// Rows 0..rows-1 of sequence b (tokens already in seq_tok) through the target (all layers) or the
+// draft (kept layers), filling that model's cache; no logits.  Per layer: activation image with the
+// norm folded in -> QKV on tcgen05 (epilogue: RoPE, K/V into the cache, q) -> causal attention over
+// the prompt -> O-projection + residual -> gate/up + SwiGLU -> down-projection + residual.
+//
+// The draft shares the target's work where it is the same work: the layers in front of the first
+// pruned layer see the same tokens through the same weights, so their K/V ARE the target's.  The
+// target's pass leaves the residual rows at that point in `h_fork`; the draft copies the K/V of
+// those layers and runs only the kept layers behind the fork.
+int dense_layer(sdfp_ctx* c, const KvCache& kv, int l, int b, int rows) {
+  const sdfp_config& g = c->cfg;
+  const int d = g.d_model, f = g.d_ffn;
+  const LayerWeights& lw = c->layers[l];
+  EpiParams qkv = base_epi(c, EPI_QKV, c->q, d);
+  qkv.kcache = kv.k[l];
+  qkv.vcache = kv.v[l];
+  CU_OK(c, run_dense_linear(c, lw.um_qkv, c->h, d, rows, d, 3 * d / 2, lw.attn_gain, qkv));
+  const float scale = 1.0f / std::sqrt((float)g.head_dim);
+  const dim3 grid((rows + kPfaQ - 1) / kPfaQ, g.n_heads);
+  const __nv_bfloat16* kc = reinterpret_cast<const __nv_bfloat16*>(kv.k[l]);
+  const __nv_bfloat16* vc = reinterpret_cast<const __nv_bfloat16*>(kv.v[l]);
+  if (g.head_dim == 128)
+    CU_OK(c, launch(c, prefill_attention_kernel<128>, grid, dim3(kPfaThreads), prefill_attention_smem<128>(), (const float*)c->q, kc,
+                    vc, c->att, rows, g.n_heads, g.max_seq, b, scale));
+  else
+    CU_OK(c, launch(c, prefill_attention_kernel<64>, grid, dim3(kPfaThreads), prefill_attention_smem<64>(), (const float*)c->q, kc, vc,
+                    c->att, rows, g.n_heads, g.max_seq, b, scale));
+  CU_OK(c, run_dense_linear(c, lw.um_wo, c->att, d, rows, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+  CU_OK(c, run_dense_linear(c, lw.um_gu, c->h, d, rows, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
+  CU_OK(c, run_dense_linear(c, lw.um_down, c->u, f, rows, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+  return 0;
+}
+
+int first_pruned_layer(const sdfp_ctx* c) {
+  for (int l = 0; l < c->cfg.n_layers; ++l)
+    if (!c->keep[l]) return l;
+  return c->cfg.n_layers;
+}
+
+// rows_t rows through the target and, when with_draft, rows_d <= rows_t rows through the draft
+int prefill_dense(sdfp_ctx* c, int b, int rows_t, int rows_d, bool with_draft) {
+  const sdfp_config& g = c->cfg;
+  const int d = g.d_model;
+  PassDesc pd{};
+  pd.kind = PASS_TOKENS;
+  pd.seq = b;
+  pd.start = 0;
+  pd.count = rows_t;
+  pd.src = c->seq_tok + (size_t)b * g.max_seq;
+  CU_OK(c, launch(c, plan_embed_kernel<__nv_bfloat16>, dim3(rows_t), dim3(128), 0, pd, (const GenState*)c->gs, (const int*)c->seq_tok,
+                  g.max_seq, (const int*)c->draft_tok, c->plan, reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, d));
+  const int fork = with_draft ? first_pruned_layer(c) : -1;  // the draft's residual rows leave the target's after this many layers
+  const size_t fork_bytes = (size_t)rows_d * d * sizeof(float);
+  if (fork == 0 && rows_d > 0) CU_OK(c, cudaMemcpyAsync(c->h_fork, c->h, fork_bytes, cudaMemcpyDeviceToDevice, c->stream));
+  for (int l = 0; l < g.n_layers; ++l) {
+    if (int r = dense_layer(c, c->cache_t, l, b, rows_t)) return r;
+    if (l + 1 == fork && rows_d > 0) CU_OK(c, cudaMemcpyAsync(c->h_fork, c->h, fork_bytes, cudaMemcpyDeviceToDevice, c->stream));
+  }
+  if (!with_draft || rows_d <= 0) return 0;
+  // K/V of the shared layers: per head one contiguous run of rows_d positions
+  const size_t pitch = (size_t)g.max_seq * g.head_dim * c->esz, width = (size_t)rows_d * g.head_dim * c->esz;
+  const size_t seq_off = (size_t)b * g.n_heads * pitch;
+  for (int l = 0; l < std::min(fork, g.n_layers); ++l) {
+    CU_OK(c, cudaMemcpy2DAsync((unsigned char*)c->cache_d.k[l] + seq_off, pitch, (const unsigned char*)c->cache_t.k[l] + seq_off, pitch,
+                               width, g.n_heads, cudaMemcpyDeviceToDevice, c->stream));
+    CU_OK(c, cudaMemcpy2DAsync((unsigned char*)c->cache_d.v[l] + seq_off, pitch, (const unsigned char*)c->cache_t.v[l] + seq_off, pitch,
+                               width, g.n_heads, cudaMemcpyDeviceToDevice, c->stream));
+  }
+  bool any = false;
+  for (int l = fork; l < g.n_layers; ++l) any = any || c->keep[l];
+  if (!any) return 0;
+  CU_OK(c, cudaMemcpyAsync(c->h, c->h_fork, fork_bytes, cudaMemcpyDeviceToDevice, c->stream));
+  pd.count = rows_d;  // the row plan of the draft's rows (positions 0..rows_d-1 are already right; rows beyond carry nothing)
+  for (int l = fork; l < g.n_layers; ++l)
+    if (c->keep[l])
+      if (int r = dense_layer(c, c->cache_d, l, b, rows_d)) return r;
   return 0;
 }
 
@@ -877,6 +1070,10 @@ extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch,
   // round always feeds the last two committed tokens)
   CU_OK(c, cudaEventRecord(c->ev[0], st));
   for (int b = 0; b < batch; ++b) {
+    if (c->use_dense && prompt_len - 1 >= kDenseMinRows) {
+      if (int r = prefill_dense(c, b, prompt_len - 1, prompt_len - 2, k > 0)) return r;
+      continue;
+    }
     if (int r = prefill_range(c, false, b, 0, prompt_len - 1)) return r;
     if (k > 0)
       if (int r = prefill_range(c, true, b, 0, prompt_len - 2)) return r;
@@ -929,6 +1126,7 @@ extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch,
   }
   CU_OK(c, cudaEventRecord(c->ev[2], st));
   if (int r = check_pass_error(c)) return r;
+  if (int r = check_dense_error(c)) return r;
 
   // results
   std::vector<int> lens(kMaxBatch);

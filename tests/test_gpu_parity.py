@@ -526,3 +526,75 @@ def test_wait_that_runs_out_returns_timeout(tiny_bf16):
     assert after.tokens == before.tokens and np.array_equal(after.stats, before.stats)
     ar = eng.sdfp_generate(prompt, 0, 24)
     assert ar.tokens == before.tokens
+
+
+# ---- the prompt pass on the tcgen05 path -------------------------------------------------------------
+
+@pytest.mark.parametrize("shape,draw,plen", [(si.TINY_BF16, "cpu", 150), (si.TINY_BF16, "cpu", 37),
+                                             (si.LLAMA7B_4L, "cuda:0", 200), (si.LLAMA13B_2L, "cuda:0", 131)])
+def test_dense_prompt_pass_fills_both_caches(shape, draw, plen):
+    """sdfp_generate sends the prompt through the dense kernels (tcgen05 linear layers, causal
+    attention over the prompt).  What they left in the target's and in the draft's cache is read
+    back through the decode kernels: the logits of the last prompt token, which attend over the
+    whole cache, must match the oracle's; so must the first generated tokens; and speculative ==
+    autoregressive as always.  The draft keeps layers behind the first pruned one, so both the
+    copied and the recomputed part of its cache are used."""
+    skip = (1,) if shape.n_layers == 2 else (1, 2)
+    eng, m, _ = make_pair(shape, skip, max_seq=plen + 40, draw_device=draw)
+    try:
+        prompt = si.make_prompts(shape.vocab, 1, plen, seed=70)
+        toks = prompt[0].tolist()
+        out = eng.sdfp_generate(prompt, 4, 12)
+        ar = eng.sdfp_generate(prompt, 0, 12)
+        assert out.tokens == ar.tokens
+        assert len(check_stream_against_oracle(m, toks, out.tokens[0])) <= 1
+        eng.sdfp_generate(prompt, 4, 1)                       # caches: target 0..P-2, draft 0..P-3 from the dense pass
+        ref = orc.forward_nocache(m, toks).detach().numpy()
+        got = eng.sdfp_forward_logits(toks[plen - 1:], plen - 1)
+        assert rel_l2(got[0], ref[plen - 1]) < 1e-2
+        kept = orc.keep_layers(shape.n_layers, skip)
+        ref_d = orc.forward_nocache(m, toks, kept).detach().numpy()
+        got_d = eng.sdfp_forward_logits(toks[plen - 2:], plen - 2, draft=True)
+        assert rel_l2(got_d[0], ref_d[plen - 2]) < 1e-2 and rel_l2(got_d[1], ref_d[plen - 1]) < 1e-2
+        # the chunked prompt pass (decode kernels, SDFP_FLAG_NO_DENSE) agrees closely
+        e2, _, _ = make_pair(shape, skip, max_seq=plen + 40, draw_device=draw, flags=pkg.FLAG_NO_DENSE)
+        try:
+            e2.sdfp_generate(prompt, 4, 1)
+            alt = e2.sdfp_forward_logits(toks[plen - 1:], plen - 1)
+            alt_d = e2.sdfp_forward_logits(toks[plen - 2:], plen - 2, draft=True)
+        finally:
+            e2.close()
+        assert rel_l2(got[0], alt[0]) < 2e-3 and rel_l2(got_d, alt_d) < 2e-3
+    finally:
+        eng.close()
+
+
+def test_dense_prompt_pass_first_layer_pruned():
+    """A draft without layer 0 shares nothing with the target: its whole prompt pass is its own."""
+    shape = si.TINY_BF16
+    eng, m, _ = make_pair(shape, (0, 2), max_seq=160)
+    try:
+        prompt = si.make_prompts(shape.vocab, 1, 100, seed=71)
+        toks = prompt[0].tolist()
+        out = eng.sdfp_generate(prompt, 3, 10)
+        assert out.tokens == eng.sdfp_generate(prompt, 0, 10).tokens
+        eng.sdfp_generate(prompt, 3, 1)
+        ref_d = orc.forward_nocache(m, toks, [1, 3]).detach().numpy()
+        got_d = eng.sdfp_forward_logits(toks[98:], 98, draft=True)
+        assert rel_l2(got_d[1], ref_d[99]) < 1e-2
+    finally:
+        eng.close()
+
+
+def test_wide_context_without_dense_path():
+    """SDFP_FLAG_NO_DENSE keeps wide contexts on the mma.sync kernels; same guarantees."""
+    eng, m, _ = make_pair(si.TINY_BF16, (1, 2), max_seq=160, max_batch=4, k_max=4, flags=pkg.FLAG_NO_DENSE)
+    try:
+        prompts = si.make_prompts(m.vocab, 4, 24, seed=54)
+        out = eng.sdfp_generate(prompts, 4, 30)
+        assert out.tokens == eng.sdfp_generate(prompts, 0, 30).tokens
+        for b in range(4):
+            assert eng.sdfp_generate(prompts[b:b + 1], 4, 30).tokens[0] == out.tokens[b]
+            check_stream_against_oracle(m, prompts[b].tolist(), out.tokens[b])
+    finally:
+        eng.close()
