@@ -42,6 +42,12 @@ design notes of the repository):
       the draft, so the next round's first draft call feeds two tokens.
   R9  Acceptance rate α = Σ accepted / Σ drafted over the run; a round's
       `committed` counts tokens appended after truncation to max_new / EOS.
+  R10 Sub-layer pruning (Section IV-A, implementation details: attention layers and FFN
+      layers are pruned at separate ratios): a decoder layer is two residual blocks,
+      h += Attn(norm(h)) and h += FFN(norm(h)); the draft may drop either one on its
+      own, and a dropped block is the identity on the residual stream.  `layers` lists
+      the layers whose attention block runs, `ffn_layers` those whose FFN block runs
+      (None = the same list: whole layers, as in Algorithm 1).
 
 Pins: see tests/test_oracle_*.py.  The absolute values of the forward pass are
 pinned by an independently written no-cache recomputation, hand-computable
@@ -125,35 +131,42 @@ class Model:
 # O4: brute force — whole sequence recomputed from scratch, no cache
 # ----------------------------------------------------------------------------
 
-def forward_nocache(m: Model, tokens: Sequence[int], layers: Optional[Sequence[int]] = None) -> torch.Tensor:
+def forward_nocache(m: Model, tokens: Sequence[int], layers: Optional[Sequence[int]] = None,
+                    ffn_layers: Optional[Sequence[int]] = None) -> torch.Tensor:
     """Logits [T, vocab] for every position of `tokens`, recomputing everything.
 
     `layers` = the layers that run (None = all = the target); the others are
     the identity on the residual stream (Algorithm 1: draft = layers removed).
+    `ffn_layers` (R10) = the layers whose FFN block runs when that differs from
+    the layers whose attention block runs.
     Written with torch ops that autograd understands (the FIT oracle
     differentiates through it).
     """
     T = len(tokens)
     H, hd = m.n_heads, m.head_dim
-    run = range(m.n_layers) if layers is None else layers
+    attn_run = set(range(m.n_layers) if layers is None else layers)
+    ffn_run = attn_run if ffn_layers is None else set(ffn_layers)
+    run = sorted(attn_run | ffn_run)
     tok = torch.tensor(list(tokens), dtype=torch.long)
     h = m.w["tok_embed"].to(m.dtype)[tok]
     cos, sin = rope_angles(hd, m.rope_theta, range(T), m.dtype)
     future = torch.triu(torch.ones(T, T, dtype=torch.bool), diagonal=1)
     for l in run:
         lw = m.w["layers"][l]
-        x = rmsnorm(h, lw["attn_norm"].to(m.dtype), m.rms_eps)
-        q = apply_rope(_lin(x, lw["wq"]).view(T, H, hd), cos, sin)
-        k = apply_rope(_lin(x, lw["wk"]).view(T, H, hd), cos, sin)
-        v = _lin(x, lw["wv"]).view(T, H, hd)
-        k, v = _store_round(k, m.kv_bf16), _store_round(v, m.kv_bf16)
-        s = torch.einsum("thd,shd->hts", q, k) / math.sqrt(hd)
-        s = s.masked_fill(future[None], float("-inf"))
-        p = torch.softmax(s, dim=-1)
-        a = torch.einsum("hts,shd->thd", p, v).reshape(T, H * hd)
-        h = h + _lin(a, lw["wo"])
-        x = rmsnorm(h, lw["ffn_norm"].to(m.dtype), m.rms_eps)
-        h = h + _lin(silu(_lin(x, lw["w_gate"])) * _lin(x, lw["w_up"]), lw["w_down"])
+        if l in attn_run:
+            x = rmsnorm(h, lw["attn_norm"].to(m.dtype), m.rms_eps)
+            q = apply_rope(_lin(x, lw["wq"]).view(T, H, hd), cos, sin)
+            k = apply_rope(_lin(x, lw["wk"]).view(T, H, hd), cos, sin)
+            v = _lin(x, lw["wv"]).view(T, H, hd)
+            k, v = _store_round(k, m.kv_bf16), _store_round(v, m.kv_bf16)
+            s = torch.einsum("thd,shd->hts", q, k) / math.sqrt(hd)
+            s = s.masked_fill(future[None], float("-inf"))
+            p = torch.softmax(s, dim=-1)
+            a = torch.einsum("hts,shd->thd", p, v).reshape(T, H * hd)
+            h = h + _lin(a, lw["wo"])
+        if l in ffn_run:
+            x = rmsnorm(h, lw["ffn_norm"].to(m.dtype), m.rms_eps)
+            h = h + _lin(silu(_lin(x, lw["w_gate"])) * _lin(x, lw["w_up"]), lw["w_down"])
     return _lin(rmsnorm(h, m.w["final_norm"].to(m.dtype), m.rms_eps), m.w["lm_head"])
 
 
@@ -170,9 +183,11 @@ class CachedLM:
     are simply never read again before being rewritten.
     """
 
-    def __init__(self, m: Model, layers: Optional[Sequence[int]] = None, max_seq: int = 4096):
+    def __init__(self, m: Model, layers: Optional[Sequence[int]] = None, max_seq: int = 4096,
+                 ffn_layers: Optional[Sequence[int]] = None):
         self.m = m
-        self.layers = list(range(m.n_layers)) if layers is None else list(layers)
+        self.layers = list(range(m.n_layers)) if layers is None else list(layers)   # attention blocks that run
+        self.ffn_layers = set(self.layers if ffn_layers is None else ffn_layers)    # FFN blocks that run (R10)
         self.max_seq = max_seq
         self.k = {l: torch.zeros(max_seq, m.n_heads, m.head_dim, dtype=m.dtype) for l in self.layers}
         self.v = {l: torch.zeros(max_seq, m.n_heads, m.head_dim, dtype=m.dtype) for l in self.layers}
@@ -191,23 +206,25 @@ class CachedLM:
         key_pos = torch.arange(start + T)
         row_pos = torch.arange(start, start + T)
         hidden = key_pos[None, :] > row_pos[:, None]            # [T, start+T]
-        for l in self.layers:
+        for l in sorted(set(self.layers) | self.ffn_layers):
             lw = m.w["layers"][l]
-            x = rmsnorm(h, lw["attn_norm"].to(m.dtype), m.rms_eps)
-            q = apply_rope(_lin(x, lw["wq"]).view(T, H, hd), cos, sin)
-            k = apply_rope(_lin(x, lw["wk"]).view(T, H, hd), cos, sin)
-            v = _lin(x, lw["wv"]).view(T, H, hd)
-            self.k[l][start:start + T] = _store_round(k, m.kv_bf16)
-            self.v[l][start:start + T] = _store_round(v, m.kv_bf16)
-            K = self.k[l][:start + T]
-            V = self.v[l][:start + T]
-            s = torch.einsum("thd,shd->hts", q, K) / math.sqrt(hd)
-            s = s.masked_fill(hidden[None], float("-inf"))
-            p = torch.softmax(s, dim=-1)
-            a = torch.einsum("hts,shd->thd", p, V).reshape(T, H * hd)
-            h = h + _lin(a, lw["wo"])
-            x = rmsnorm(h, lw["ffn_norm"].to(m.dtype), m.rms_eps)
-            h = h + _lin(silu(_lin(x, lw["w_gate"])) * _lin(x, lw["w_up"]), lw["w_down"])
+            if l in self.k:
+                x = rmsnorm(h, lw["attn_norm"].to(m.dtype), m.rms_eps)
+                q = apply_rope(_lin(x, lw["wq"]).view(T, H, hd), cos, sin)
+                k = apply_rope(_lin(x, lw["wk"]).view(T, H, hd), cos, sin)
+                v = _lin(x, lw["wv"]).view(T, H, hd)
+                self.k[l][start:start + T] = _store_round(k, m.kv_bf16)
+                self.v[l][start:start + T] = _store_round(v, m.kv_bf16)
+                K = self.k[l][:start + T]
+                V = self.v[l][:start + T]
+                s = torch.einsum("thd,shd->hts", q, K) / math.sqrt(hd)
+                s = s.masked_fill(hidden[None], float("-inf"))
+                p = torch.softmax(s, dim=-1)
+                a = torch.einsum("hts,shd->thd", p, V).reshape(T, H * hd)
+                h = h + _lin(a, lw["wo"])
+            if l in self.ffn_layers:
+                x = rmsnorm(h, lw["ffn_norm"].to(m.dtype), m.rms_eps)
+                h = h + _lin(silu(_lin(x, lw["w_gate"])) * _lin(x, lw["w_up"]), lw["w_down"])
         return _lin(rmsnorm(h, m.w["final_norm"].to(m.dtype), m.rms_eps), m.w["lm_head"])
 
 

@@ -351,3 +351,30 @@ def test_bf16_model_kv_rounding():
     assert torch.equal(k, k.to(torch.bfloat16).to(torch.float32))
     full = o.forward_nocache(m, toks)
     assert ((inc - full).norm() / full.norm()).item() < 1e-4
+
+
+def test_skipped_sub_blocks_equal_zeroed_output_projections():
+    """Sub-layer pruning (reading R10): dropping a layer's attention block is the same function as
+    zeroing its wo, dropping its FFN block the same as zeroing its w_down, independently of each
+    other; no-cache and cached forward agree; and the two blocks are not interchangeable."""
+    m = _tiny_model(dtype=torch.float64)
+    toks = si.make_prompts(m.vocab, 1, 12, seed=4)[0].tolist()
+    attn_keep, ffn_keep = [0, 2, 3], [0, 1, 3]          # layer 1 loses attention, layer 2 loses its FFN
+    got = o.forward_nocache(m, toks, attn_keep, ffn_keep)
+    import copy
+    w2 = copy.deepcopy(m.w)
+    w2["layers"][1]["wo"].zero_()
+    w2["layers"][2]["w_down"].zero_()
+    m2 = o.Model.from_shape(si.TINY, w2, dtype=torch.float64)
+    want = o.forward_nocache(m2, toks)
+    assert torch.allclose(got, want, rtol=1e-10, atol=1e-12)
+    lm = o.CachedLM(m, attn_keep, max_seq=16, ffn_layers=ffn_keep)
+    a = lm.feed(toks[:7], 0)
+    b = lm.feed(toks[7:], 7)
+    assert torch.allclose(torch.cat([a, b]), want, rtol=1e-9, atol=1e-11)
+    assert sorted(lm.k.keys()) == attn_keep                 # a cache only for the attention blocks that run
+    # swapping the roles gives another function
+    other = o.forward_nocache(m, toks, ffn_keep, attn_keep)
+    assert not torch.allclose(other, want, rtol=1e-3, atol=1e-6)
+    # whole layers are the special case of equal lists
+    assert torch.equal(o.forward_nocache(m, toks, [0, 3], [0, 3]), o.forward_nocache(m, toks, [0, 3]))
