@@ -40,6 +40,8 @@ WORKLOADS = {
     "c2-7b-greedy-k4": (si.LLAMA7B, 12, 4, 512, 256, 0.0, 1),       # the configuration the metric is quoted on
     "c3-7b-sampled-k6": (si.LLAMA7B, 12, 6, 512, 256, 1.0, 1),      # rejection sampling, residual resampling
     "c4-13b-greedy-k4": (si.LLAMA13B, 16, 4, 2048, 512, 0.0, 1),    # long KV cache
+    # the paper's own 13B setting: 50 % of the attention blocks and 35 % of the FFN blocks pruned
+    "c4-13b-sublayer-k4": (si.LLAMA13B, (20, 14), 4, 2048, 512, 0.0, 1),
     "c1-tiny-greedy-k4": (si.TINY, 2, 4, 16, 64, 0.0, 1),
     "7b-4layers-greedy-k4": (si.LLAMA7B_4L, 2, 4, 64, 64, 0.0, 1),
     "7b-4layers-b8-greedy-k4": (si.LLAMA7B_4L, 2, 4, 64, 64, 0.0, 8),
@@ -117,7 +119,15 @@ class ClockSampler:
         return out
 
 
-def oracle_sample(shape, w_cpu, skip, k, prompt_len_sample, new_tokens, n_threads, temperature=0.0):
+def skip_sets(shape, n_skip):
+    """(attention blocks, FFN blocks) the draft drops; an int means whole layers."""
+    if isinstance(n_skip, tuple):
+        return (si.choose_skip_layers(shape.n_layers, n_skip[0]), si.choose_skip_layers(shape.n_layers, n_skip[1]))
+    s = si.choose_skip_layers(shape.n_layers, n_skip)
+    return s, s
+
+
+def oracle_sample(shape, w_cpu, skip, k, prompt_len_sample, new_tokens, n_threads, temperature=0.0, skip_ffn=None):
     """Times the CPU oracle, as it stands, on a bounded sample: speculative greedy decode of
     `new_tokens` tokens after a `prompt_len_sample`-token prompt.  Returns tokens/s of the
     decode part (prompt pass excluded, like the GPU number) and a description."""
@@ -128,7 +138,8 @@ def oracle_sample(shape, w_cpu, skip, k, prompt_len_sample, new_tokens, n_thread
     prompt = si.make_prompts(shape.vocab, 1, prompt_len_sample)[0].tolist()
     cap = prompt_len_sample + new_tokens + k + 2
     tgt = orc.CachedLM(m, max_seq=cap)
-    drf = orc.CachedLM(m, orc.keep_layers(shape.n_layers, skip), max_seq=cap)
+    drf = orc.CachedLM(m, orc.keep_layers(shape.n_layers, skip), max_seq=cap,
+                       ffn_layers=None if skip_ffn is None else orc.keep_layers(shape.n_layers, skip_ffn))
     t0 = time.perf_counter()
     tgt.feed(prompt[:-1], 0)
     drf.feed(prompt[:-1], 0)
@@ -167,17 +178,17 @@ def run_reference(args, workload):
     """--impl reference: the oracle on the host cores (rank 0 only)."""
     import torch
     shape, n_skip, k, plen, n_new, temp, _batch = WORKLOADS[workload]
-    skip = si.choose_skip_layers(shape.n_layers, n_skip)
+    skip, skip_ffn = skip_sets(shape, n_skip)
     cores = os.cpu_count() or 1
     big = shape.n_params() > 1e9
     dev = "cuda:0" if (big and torch.cuda.is_available()) else "cpu"
-    w = si.make_weights(shape, skip, device=dev)
+    w = si.make_weights(shape, skip, device=dev, skip_ffn=skip_ffn)
     w_cpu = si.weights_to(w, "cpu")
     del w
     sample_prompt, sample_new = (32, 8) if big else (plen, n_new)
     vals, secs = [], []
     for i in range(args.warmup + args.steps):
-        v, dt, _, _ = oracle_sample(shape, w_cpu, skip, k, sample_prompt, sample_new, cores, temp)
+        v, dt, _, _ = oracle_sample(shape, w_cpu, skip, k, sample_prompt, sample_new, cores, temp, skip_ffn)
         if i >= args.warmup:
             vals.append(v)
             secs.append(dt)
@@ -224,11 +235,11 @@ def main():
     pkg.build_library()
 
     shape, n_skip, k, plen, n_new, temp, batch = WORKLOADS[args.workload]
-    skip = si.choose_skip_layers(shape.n_layers, n_skip)
+    skip, skip_ffn = skip_sets(shape, n_skip)
     dev = f"cuda:{local_rank}"
-    w = si.make_weights(shape, skip, device=dev)
+    w = si.make_weights(shape, skip, device=dev, skip_ffn=skip_ffn)
     eng = pkg.Sdfp(shape, w, max_seq=plen + n_new + 16, max_batch=batch, k_max=8, flags=args.flags)
-    eng.sdfp_set_draft_layers(si.keep_mask(shape.n_layers, skip))
+    eng.sdfp_set_draft_sublayers(si.keep_mask(shape.n_layers, skip), si.keep_mask(shape.n_layers, skip_ffn))
     want_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
     w_cpu = si.weights_to(w, "cpu") if want_cpu else None
     del w
@@ -304,8 +315,8 @@ def main():
             per_kernel[name] = {"us": round(ms * 1e3, 1), "GB/s": round(nbytes / ms / 1e6, 1),
                                 "bytes": int(nbytes), "frac_of_peak": round(nbytes / ms / 1e6 / peak, 3)}
         dom_ms, dom_bytes = eng.sdfp_time_pass(True, 1, mid, 48)
-        dom_name = "pass_kernel (draft pass: %d of %d layers + lm-head, M=1, context %d)" % (
-            shape.n_layers - len(skip), shape.n_layers, mid)
+        dom_name = "pass_kernel (draft pass: %d attention and %d FFN blocks of %d layers + lm-head, M=1, context %d)" % (
+            shape.n_layers - len(skip), shape.n_layers - len(skip_ffn), shape.n_layers, mid)
     else:
         names = ["qkv", "o_proj", "gate_up", "down", "lm_head"]
         for rows in (batch, batch * (k + 1)):
@@ -328,7 +339,7 @@ def main():
         cores = os.cpu_count() or 1
         big = shape.n_params() > 1e9
         sp, sn = (32, 8) if big else (plen, n_new)
-        v, dt, pre_dt, _ = oracle_sample(shape, w_cpu, skip, k, sp, sn, cores, temp)
+        v, dt, pre_dt, _ = oracle_sample(shape, w_cpu, skip, k, sp, sn, cores, temp, skip_ffn)
         cpu_baseline = {"value": v, "unit": "tokens/s", "cores": cores, "kind": "oracle",
                         "sample": f"speculative greedy decode of {sn} tokens after a {sp}-token prompt, k={k}, "
                                   f"{dt:.1f} s (+ {pre_dt:.1f} s prompt pass)"}
@@ -339,7 +350,7 @@ def main():
             "warmup": args.warmup, "ms_per_step": step_ms_max, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16" if shape.dtype == "bf16" else "f32", "data": "synthetic",
             "config": {"workload": args.workload, "shape": shape.name, "batch": batch, "prompt_len": plen,
-                       "max_new": n_new, "k": k, "skip_layers": skip,
+                       "max_new": n_new, "k": k, "skip_layers": skip, "skip_ffn_blocks": skip_ffn,
                        "decoding": "greedy" if temp == 0.0 else "sampled, temperature %g, Philox seed %d" % (temp, SEED),
                        "l2": "inputs larger than L2 (weights %.1f GB per pass)" % (shape.n_params() * 2 / 1e9)
                        if shape.dtype == "bf16" else "tiny model: launch-bound, weights fit in L2",

@@ -140,6 +140,17 @@ int sdfp_create(const sdfp_config *cfg, const sdfp_weights *w, void *cuda_stream
 int sdfp_set_draft_layers(sdfp_ctx *ctx, const uint8_t *keep_mask);
 
 /*
+ * The same at sub-layer granularity (Section IV-A, implementation details: attention layers and
+ * FFN layers are pruned at separate ratios, e.g. 50 % and 35 % for the 13B model).  A decoder
+ * layer is two residual blocks, h += Attn(norm(h)) and h += FFN(norm(h)); keep_attn and keep_ffn
+ * are HOST arrays of n_layers bytes each, 1 = the draft runs that block, 0 = the block is the
+ * identity for the draft.  At least one block must be kept.  The draft's KV cache is used for
+ * the layers whose attention block runs.  sdfp_set_draft_layers(m) is
+ * sdfp_set_draft_sublayers(m, m).  Takes effect at the next sdfp_generate.
+ */
+int sdfp_set_draft_sublayers(sdfp_ctx *ctx, const uint8_t *keep_attn, const uint8_t *keep_ffn);
+
+/*
  * Generate (Algorithm 1, Stage B).  Synchronous: returns when the outputs are
  * in host memory.
  *   prompts     host int32 [batch, prompt_len], ids in [0, vocab); prompt_len >= 1

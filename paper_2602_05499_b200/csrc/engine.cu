@@ -69,7 +69,7 @@ struct sdfp_ctx {
   float* final_gain = nullptr;
   float *rope_cos = nullptr, *rope_sin = nullptr;
   KvCache cache_t, cache_d;
-  std::vector<uint8_t> keep;
+  std::vector<uint8_t> keep_attn, keep_ffn;  // draft: which attention blocks and which FFN blocks run
 
   // activations / scratch
   float *h = nullptr, *q = nullptr, *att = nullptr, *u = nullptr, *logits = nullptr;
@@ -322,28 +322,31 @@ int build_program(sdfp_ctx* c, bool draft, StageDesc** dev, int* n_out) {
   const KvCache& kv = draft ? c->cache_d : c->cache_t;
   std::vector<StageDesc> prog;
   for (int l = 0; l < g.n_layers; ++l) {
-    if (draft && !c->keep[l]) continue;
     const LayerWeights& lw = c->layers[l];
-    EpiParams qkv = base_epi(c, EPI_QKV, c->q, d);
-    qkv.kcache = kv.k[l];
-    qkv.vcache = kv.v[l];
-    prog.push_back(linear_desc(lw.qkv, c->h, d, 3 * d / 2, lw.attn_gain, qkv));
-    // the embedding rows come from another kernel: the first norm of a pass sums its rows itself
-    if (prog.size() == 1) prog.back().rms_mode = RMS_DIRECT;
-    StageDesc at{};
-    at.kind = ST_ATTN;
-    at.X = c->q;
-    at.ep = base_epi(c, EPI_RESID, nullptr, d);
-    at.ep.kcache = kv.k[l];
-    at.ep.vcache = kv.v[l];
-    prog.push_back(at);
-    // the O-projection reads the attention output as kAttnSplits partials per (row, head)
-    prog.push_back(linear_desc(lw.wo, nullptr, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
-    prog.back().x_mode = X_ATTN_FOLD;
-    prog.push_back(linear_desc(lw.gu, c->h, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
-    prog.push_back(linear_desc(lw.down, c->u, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+    if (!draft || c->keep_attn[l]) {  // the attention block: h += Wo * Attn(norm(h))
+      EpiParams qkv = base_epi(c, EPI_QKV, c->q, d);
+      qkv.kcache = kv.k[l];
+      qkv.vcache = kv.v[l];
+      prog.push_back(linear_desc(lw.qkv, c->h, d, 3 * d / 2, lw.attn_gain, qkv));
+      StageDesc at{};
+      at.kind = ST_ATTN;
+      at.X = c->q;
+      at.ep = base_epi(c, EPI_RESID, nullptr, d);
+      at.ep.kcache = kv.k[l];
+      at.ep.vcache = kv.v[l];
+      prog.push_back(at);
+      // the O-projection reads the attention output as kAttnSplits partials per (row, head)
+      prog.push_back(linear_desc(lw.wo, nullptr, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+      prog.back().x_mode = X_ATTN_FOLD;
+    }
+    if (!draft || c->keep_ffn[l]) {   // the FFN block: h += Wdown * SwiGLU(norm(h))
+      prog.push_back(linear_desc(lw.gu, c->h, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
+      prog.push_back(linear_desc(lw.down, c->u, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+    }
   }
   prog.push_back(linear_desc(c->lm_head, c->h, d, g.vocab / 2, c->final_gain, base_epi(c, EPI_LOGITS, c->logits, g.vocab)));
+  // the embedding rows come from another kernel: the first norm of a pass sums its rows itself
+  prog.front().rms_mode = RMS_DIRECT;
   for (StageDesc& sd : prog) sd.ssq_groups = resid_groups;
   if (*dev == nullptr)
     if (int r = dev_alloc(c, dev, (size_t)5 * g.n_layers + 1)) return r;
@@ -479,19 +482,19 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
   if (whole_pass && rows > kPassMaxRows) return fail(c, SDFP_ESTATE, "a pass of %d rows reached the whole-pass kernel", rows);
   if (whole_pass) CU_OK(c, run_pass(c, draft, rows, attn_rows_per_seq, decide != DECIDE_NONE));
   for (int l = 0; l < g.n_layers && !whole_pass; ++l) {
-    if (draft && !c->keep[l]) continue;  // Algorithm 1: pruned layers are removed from the draft
+    // Algorithm 1: pruned layers are removed from the draft, attention and FFN blocks separately
+    const bool run_attn = !draft || c->keep_attn[l], run_ffn = !draft || c->keep_ffn[l];
     const LayerWeights& lw = c->layers[l];
-    {
+    if (run_attn) {
       LinearCall lc{lw.qkv, c->h, d, rows, d, 3 * d / 2, lw.attn_gain, base_epi(c, EPI_QKV, c->q, d)};
       lc.ep.kcache = kv.k[l];
       lc.ep.vcache = kv.v[l];
       CU_OK(c, run_linear(c, lc));
+      CU_OK(c, run_attention(c, kv, l, rows, attn_rows_per_seq, n_chunks));
+      LinearCall lo{lw.wo, c->att, d, rows, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)};
+      CU_OK(c, run_linear(c, lo));
     }
-    CU_OK(c, run_attention(c, kv, l, rows, attn_rows_per_seq, n_chunks));
-    {
-      LinearCall lc{lw.wo, c->att, d, rows, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)};
-      CU_OK(c, run_linear(c, lc));
-    }
+    if (!run_ffn) continue;
     {
       LinearCall lc{lw.gu, c->h, d, rows, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)};
       CU_OK(c, run_linear(c, lc));
@@ -636,16 +639,21 @@ int alloc_cache(sdfp_ctx* c, KvCache& kv) {
   return 0;
 }
 
-int64_t layer_weight_bytes(const sdfp_ctx* c) {
-  const int64_t d = c->cfg.d_model, f = c->cfg.d_ffn;
-  return (4 * d * d + 3 * d * f) * (int64_t)c->esz;
-}
+int64_t attn_block_bytes(const sdfp_ctx* c) { return 4LL * c->cfg.d_model * c->cfg.d_model * (int64_t)c->esz; }
+int64_t ffn_block_bytes(const sdfp_ctx* c) { return 3LL * c->cfg.d_model * c->cfg.d_ffn * (int64_t)c->esz; }
 int64_t lm_head_bytes(const sdfp_ctx* c) { return (int64_t)c->cfg.vocab * c->cfg.d_model * (int64_t)c->esz; }
-int kept_layers(const sdfp_ctx* c) {
+int kept_blocks(const std::vector<uint8_t>& keep) {
   int n = 0;
-  for (uint8_t x : c->keep) n += x ? 1 : 0;
+  for (uint8_t x : keep) n += x ? 1 : 0;
   return n;
 }
+// weight bytes one pass of the draft / of the target has to read, lm-head excluded
+int64_t pass_weight_bytes(const sdfp_ctx* c, bool draft) {
+  const int64_t na = draft ? kept_blocks(c->keep_attn) : c->cfg.n_layers, nf = draft ? kept_blocks(c->keep_ffn) : c->cfg.n_layers;
+  return na * attn_block_bytes(c) + nf * ffn_block_bytes(c);
+}
+// layers whose K/V a pass reads and writes
+int64_t pass_kv_layers(const sdfp_ctx* c, bool draft) { return draft ? kept_blocks(c->keep_attn) : c->cfg.n_layers; }
 
 }  // namespace
 
@@ -719,7 +727,8 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   c->use_pdl = !(g.flags & SDFP_FLAG_NO_PDL);
   c->use_graph = !(g.flags & SDFP_FLAG_NO_GRAPH);
   c->L.pdl = c->use_pdl;
-  c->keep.assign(g.n_layers, 1);
+  c->keep_attn.assign(g.n_layers, 1);
+  c->keep_ffn.assign(g.n_layers, 1);
   int dev = 0;
   cudaDeviceProp prop;
   if (cudaGetDevice(&dev) != cudaSuccess || cudaGetDeviceProperties(&prop, dev) != cudaSuccess) {
@@ -843,23 +852,34 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   return 0;
 }
 
-extern "C" int sdfp_set_draft_layers(sdfp_ctx* c, const uint8_t* keep_mask) {
+extern "C" int sdfp_set_draft_sublayers(sdfp_ctx* c, const uint8_t* keep_attn, const uint8_t* keep_ffn) {
   if (!c) return SDFP_EINVAL;
-  if (!keep_mask) return fail(c, SDFP_EINVAL, "keep_mask is NULL");
-  if (int r = check_device(c, "sdfp_set_draft_layers")) return r;
+  if (!keep_attn || !keep_ffn) return fail(c, SDFP_EINVAL, "keep mask is NULL");
+  if (int r = check_device(c, "sdfp_set_draft_sublayers")) return r;
+  const int L = c->cfg.n_layers;
   int kept = 0;
-  for (int l = 0; l < c->cfg.n_layers; ++l) kept += keep_mask[l] ? 1 : 0;
-  if (kept == 0) return fail(c, SDFP_EINVAL, "the draft must keep at least one layer");
+  for (int l = 0; l < L; ++l) kept += (keep_attn[l] ? 1 : 0) + (keep_ffn[l] ? 1 : 0);
+  if (kept == 0) return fail(c, SDFP_EINVAL, "the draft must keep at least one block");
   bool same = true;
-  for (int l = 0; l < c->cfg.n_layers; ++l) same = same && ((keep_mask[l] != 0) == (c->keep[l] != 0));
+  for (int l = 0; l < L; ++l)
+    same = same && ((keep_attn[l] != 0) == (c->keep_attn[l] != 0)) && ((keep_ffn[l] != 0) == (c->keep_ffn[l] != 0));
   if (!same) {
-    for (int l = 0; l < c->cfg.n_layers; ++l) c->keep[l] = keep_mask[l] ? 1 : 0;
-    for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);  // captured rounds baked the old layer set in
+    for (int l = 0; l < L; ++l) {
+      c->keep_attn[l] = keep_attn[l] ? 1 : 0;
+      c->keep_ffn[l] = keep_ffn[l] ? 1 : 0;
+    }
+    for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);  // captured rounds baked the old block set in
     c->graphs.clear();
     CU_OK(c, cudaStreamSynchronize(c->stream));
     if (int r = build_programs(c)) return r;
   }
   return 0;
+}
+
+extern "C" int sdfp_set_draft_layers(sdfp_ctx* c, const uint8_t* keep_mask) {
+  if (!c) return SDFP_EINVAL;
+  if (!keep_mask) return fail(c, SDFP_EINVAL, "keep_mask is NULL");
+  return sdfp_set_draft_sublayers(c, keep_mask, keep_mask);
 }
 
 namespace {
@@ -956,10 +976,16 @@ int prefill_range(sdfp_ctx* c, bool draft, int b, int from, int to) {
 // pruned layer see the same tokens through the same weights, so their K/V ARE the target's.  The
 // target's pass leaves the residual rows at that point in `h_fork`; the draft copies the K/V of
 // those layers and runs only the kept layers behind the fork.
-int dense_layer(sdfp_ctx* c, const KvCache& kv, int l, int b, int rows) {
+int dense_layer(sdfp_ctx* c, const KvCache& kv, int l, int b, int rows, bool run_attn, bool run_ffn) {
   const sdfp_config& g = c->cfg;
   const int d = g.d_model, f = g.d_ffn;
   const LayerWeights& lw = c->layers[l];
+  if (run_ffn && !run_attn) {
+    CU_OK(c, run_dense_linear(c, lw.um_gu, c->h, d, rows, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
+    CU_OK(c, run_dense_linear(c, lw.um_down, c->u, f, rows, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+    return 0;
+  }
+  if (!run_attn) return 0;
   EpiParams qkv = base_epi(c, EPI_QKV, c->q, d);
   qkv.kcache = kv.k[l];
   qkv.vcache = kv.v[l];
@@ -975,6 +1001,7 @@ int dense_layer(sdfp_ctx* c, const KvCache& kv, int l, int b, int rows) {
     CU_OK(c, launch(c, prefill_attention_kernel<64>, grid, dim3(kPfaThreads), prefill_attention_smem<64>(), (const float*)c->q, kc, vc,
                     c->att, rows, g.n_heads, g.max_seq, b, scale));
   CU_OK(c, run_dense_linear(c, lw.um_wo, c->att, d, rows, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+  if (!run_ffn) return 0;
   CU_OK(c, run_dense_linear(c, lw.um_gu, c->h, d, rows, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
   CU_OK(c, run_dense_linear(c, lw.um_down, c->u, f, rows, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
   return 0;
@@ -982,7 +1009,7 @@ int dense_layer(sdfp_ctx* c, const KvCache& kv, int l, int b, int rows) {
 
 int first_pruned_layer(const sdfp_ctx* c) {
   for (int l = 0; l < c->cfg.n_layers; ++l)
-    if (!c->keep[l]) return l;
+    if (!c->keep_attn[l] || !c->keep_ffn[l]) return l;  // the first layer of which the draft drops a block
   return c->cfg.n_layers;
 }
 
@@ -1002,7 +1029,7 @@ int prefill_dense(sdfp_ctx* c, int b, int rows_t, int rows_d, bool with_draft) {
   const size_t fork_bytes = (size_t)rows_d * d * sizeof(float);
   if (fork == 0 && rows_d > 0) CU_OK(c, cudaMemcpyAsync(c->h_fork, c->h, fork_bytes, cudaMemcpyDeviceToDevice, c->stream));
   for (int l = 0; l < g.n_layers; ++l) {
-    if (int r = dense_layer(c, c->cache_t, l, b, rows_t)) return r;
+    if (int r = dense_layer(c, c->cache_t, l, b, rows_t, true, true)) return r;
     if (l + 1 == fork && rows_d > 0) CU_OK(c, cudaMemcpyAsync(c->h_fork, c->h, fork_bytes, cudaMemcpyDeviceToDevice, c->stream));
   }
   if (!with_draft || rows_d <= 0) return 0;
@@ -1016,13 +1043,12 @@ int prefill_dense(sdfp_ctx* c, int b, int rows_t, int rows_d, bool with_draft) {
                                width, g.n_heads, cudaMemcpyDeviceToDevice, c->stream));
   }
   bool any = false;
-  for (int l = fork; l < g.n_layers; ++l) any = any || c->keep[l];
+  for (int l = fork; l < g.n_layers; ++l) any = any || c->keep_attn[l] || c->keep_ffn[l];
   if (!any) return 0;
   CU_OK(c, cudaMemcpyAsync(c->h, c->h_fork, fork_bytes, cudaMemcpyDeviceToDevice, c->stream));
   pd.count = rows_d;  // the row plan of the draft's rows (positions 0..rows_d-1 are already right; rows beyond carry nothing)
   for (int l = fork; l < g.n_layers; ++l)
-    if (c->keep[l])
-      if (int r = dense_layer(c, c->cache_d, l, b, rows_d)) return r;
+    if (int r = dense_layer(c, c->cache_d, l, b, rows_d, c->keep_attn[l] != 0, c->keep_ffn[l] != 0)) return r;
   return 0;
 }
 
@@ -1154,9 +1180,9 @@ extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch,
   t.n_draft_passes = rounds * k;
   t.n_target_passes = rounds;
   t.kernel_launches = c->launches - launches0;
-  const int64_t lw = layer_weight_bytes(c), lm = lm_head_bytes(c);
-  const int kept = kept_layers(c);
-  t.weight_bytes = (int64_t)rounds * ((int64_t)k * (kept * lw + lm) + (int64_t)g.n_layers * lw + lm);
+  const int64_t lm = lm_head_bytes(c);
+  const int64_t kept = pass_kv_layers(c, true);
+  t.weight_bytes = (int64_t)rounds * ((int64_t)k * (pass_weight_bytes(c, true) + lm) + pass_weight_bytes(c, false) + lm);
   const int64_t kv_tok = 2LL * g.d_model * (int64_t)c->esz;  // K and V of one token of one layer
   std::vector<int> n(batch, prompt_len);
   for (int r = 0; r < rounds; ++r)
@@ -1329,9 +1355,9 @@ extern "C" int sdfp_time_pass(sdfp_ctx* c, int32_t draft, int32_t rows, int32_t 
   CU_OK(c, err);
   if (int r = check_pass_error(c)) return r;
   *ms_per_launch = (float)(total / iters);
-  const int64_t layers = draft ? kept_layers(c) : g.n_layers;
+  const int64_t layers = pass_kv_layers(c, draft != 0);
   const int64_t kv_tok = 2LL * g.d_model * (int64_t)c->esz;
-  *bytes_per_launch = layers * layer_weight_bytes(c) + lm_head_bytes(c) + layers * kv_tok * ((int64_t)position + rows) +
+  *bytes_per_launch = pass_weight_bytes(c, draft != 0) + lm_head_bytes(c) + layers * kv_tok * ((int64_t)position + rows) +
                       layers * kv_tok * rows;
   return 0;
 }

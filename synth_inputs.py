@@ -108,7 +108,8 @@ def _gain(d: int, seed: int, device: str, random_gains: bool) -> torch.Tensor:
 
 
 def make_weights(shape: ModelShape, skip: Sequence[int], seed: int = MASTER_SEED,
-                 down_scale: float = 0.05, device: str = "cpu", random_gains: bool = False) -> Dict:
+                 down_scale: float = 0.05, device: str = "cpu", random_gains: bool = False,
+                 skip_ffn: Sequence[int] = None) -> Dict:
     """Random-init weights as a dict of torch tensors on `device`.
 
     Matrices are [out_features, in_features] row-major.  The draw happens on
@@ -116,11 +117,14 @@ def make_weights(shape: ModelShape, skip: Sequence[int], seed: int = MASTER_SEED
     the same seed, so a test that needs the same model on both sides draws once
     and copies).  Storage dtype follows shape.dtype.  random_gains=True replaces the
     unit RMSNorm gains by seeded draws from [0.5, 1.5) (rounded to the storage type), so
-    that a test can see whether every gain reaches the right column.
+    that a test can see whether every gain reaches the right column.  With skip_ffn given,
+    the pruned blocks are chosen per sub-layer: o_proj is scaled in the layers of `skip`
+    (attention blocks the draft drops), down_proj in the layers of `skip_ffn`.
     """
     st = torch.float32 if shape.dtype == "f32" else torch.bfloat16
     d, f, v = shape.d_model, shape.d_ffn, shape.vocab
     skip = set(int(s) for s in skip)
+    skip_ffn = skip if skip_ffn is None else set(int(s) for s in skip_ffn)
     w: Dict = {"layers": []}
     w["tok_embed"] = _normal((v, d), seed * 1000 + 1, device).to(st)
     w["lm_head"] = _normal((v, d), seed * 1000 + 2, device).to(st)
@@ -131,7 +135,7 @@ def make_weights(shape: ModelShape, skip: Sequence[int], seed: int = MASTER_SEED
         lw = {}
         for ti, name in enumerate(_TENSORS_PER_LAYER):
             t = _normal(dims[name], seed * 1000 + 10 + l * 16 + ti, device)
-            if l in skip and name in ("wo", "w_down"):
+            if (l in skip and name == "wo") or (l in skip_ffn and name == "w_down"):
                 t = t * down_scale
             lw[name] = t.to(st)
         lw["attn_norm"] = _gain(d, seed * 1000 + 10 + l * 16 + 8, device, random_gains).to(st)

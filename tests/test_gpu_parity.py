@@ -598,3 +598,56 @@ def test_wide_context_without_dense_path():
             check_stream_against_oracle(m, prompts[b].tolist(), out.tokens[b])
     finally:
         eng.close()
+
+
+# ---- sub-layer draft masks (attention and FFN blocks pruned separately) -----------------------------
+
+@pytest.mark.parametrize("shape,draw,flags", [(si.TINY, "cpu", 0), (si.TINY_BF16, "cpu", 0),
+                                              (si.TINY_BF16, "cpu", pkg.FLAG_NO_PASS_KERNEL), (si.LLAMA7B_4L, "cuda:0", 0)])
+def test_sublayer_draft_mask(shape, draw, flags):
+    """The draft drops the attention block of layers 1 and 2 and the FFN block of layer 2 only
+    (Section IV-A prunes the two kinds of sub-layer at different ratios).  Draft logits against
+    the oracle with the same two lists; speculative == autoregressive; acceptance counts
+    against the oracle's loop; a mask whose first kept block is an FFN block."""
+    skip_attn, skip_ffn = (1, 2), (2,)
+    pkg.build_library()
+    w = si.make_weights(shape, skip_attn, device=draw, skip_ffn=skip_ffn)
+    m = orc.Model.from_shape(shape, si.weights_to(w, "cpu"))
+    eng = pkg.Sdfp(shape, si.weights_to(w, "cuda:0"), max_seq=200, k_max=4, flags=flags)
+    try:
+        ka, kf = si.keep_mask(shape.n_layers, skip_attn), si.keep_mask(shape.n_layers, skip_ffn)
+        eng.sdfp_set_draft_sublayers(ka, kf)
+        la, lf = orc.keep_layers(shape.n_layers, skip_attn), orc.keep_layers(shape.n_layers, skip_ffn)
+        toks = si.make_prompts(shape.vocab, 1, 40, seed=80)[0].tolist()
+        tol = 1e-4 if shape.dtype == "f32" else 1e-2
+        lm = orc.CachedLM(m, la, max_seq=64, ffn_layers=lf)
+        got = np.concatenate([eng.sdfp_forward_logits(toks[:17], 0, draft=True), eng.sdfp_forward_logits(toks[17:], 17, draft=True)])
+        ref = lm.feed(toks, 0).numpy()
+        assert max(rel_l2(got[r], ref[r]) for r in range(40)) < tol
+        for plen in (12, 150):                       # short prompt: chunked prompt pass; long: the dense one (bf16)
+            prompt = si.make_prompts(shape.vocab, 1, plen, seed=81)
+            out = eng.sdfp_generate(prompt, 4, 24)
+            ar = eng.sdfp_generate(prompt, 0, 24)
+            assert out.tokens == ar.tokens
+            rep = check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+            ref_run = orc.spec_generate(orc.CachedLM(m, max_seq=200), orc.CachedLM(m, la, max_seq=200, ffn_layers=lf),
+                                        prompt[0].tolist(), 4, 24)
+            if not rep and ref_run.tokens == out.tokens[0] and shape.dtype == "f32":
+                assert out.stats[:, 0, 1].tolist() == [r.accepted for r in ref_run.rounds]
+        t = eng.sdfp_generate(si.make_prompts(shape.vocab, 1, 12, seed=81), 4, 24).timing
+        d, f = shape.d_model, shape.d_ffn
+        esz = 4 if shape.dtype == "f32" else 2
+        per_draft = (len(la) * 4 * d * d + len(lf) * 3 * d * f + shape.vocab * d) * esz
+        per_target = (shape.n_layers * (4 * d * d + 3 * d * f) + shape.vocab * d) * esz
+        assert t["weight_bytes"] == t["n_rounds"] * (4 * per_draft + per_target)
+        # a draft whose first block is an FFN block (layer 0 keeps only its FFN)
+        eng.sdfp_set_draft_sublayers([0, 1, 0, 1], [1, 0, 0, 1])
+        lm2 = orc.CachedLM(m, [1, 3], max_seq=64, ffn_layers=[0, 3])
+        got2 = eng.sdfp_forward_logits(toks[:9], 0, draft=True)
+        assert max(rel_l2(got2[r], r2) for r, r2 in enumerate(lm2.feed(toks[:9], 0).numpy())) < tol
+        prompt = si.make_prompts(shape.vocab, 1, 60, seed=82)
+        assert eng.sdfp_generate(prompt, 3, 16).tokens == eng.sdfp_generate(prompt, 0, 16).tokens
+        with pytest.raises(pkg.SdfpError):
+            eng.sdfp_set_draft_sublayers([0] * shape.n_layers, [0] * shape.n_layers)
+    finally:
+        eng.close()
