@@ -45,6 +45,7 @@ WORKLOADS = {
     "c1-tiny-greedy-k4": (si.TINY, 2, 4, 16, 64, 0.0, 1),
     "7b-4layers-greedy-k4": (si.LLAMA7B_4L, 2, 4, 64, 64, 0.0, 1),
     "7b-4layers-b8-greedy-k4": (si.LLAMA7B_4L, 2, 4, 64, 64, 0.0, 8),
+    "7b-4layers-b8-long-greedy-k4": (si.LLAMA7B_4L, 2, 4, 1024, 64, 0.0, 8),   # the batch-8 context length at 4 layers
 }
 # batch 8 with ragged acceptance: draft length k and share of skipped layers swept
 for _k in (2, 4, 8):

@@ -32,7 +32,26 @@ struct AttnParams {
   const int* row_seq;
   int n_heads, max_seq, n_chunks;
   float scale;       // 1/sqrt(head_dim)
+  // non-null: leave the result as bf16 hi + lo in the activation image of the O-projection on the
+  // dense path instead of fp32 rows (row block img_rb, img_kb k blocks of 64; 16-byte piece of
+  // (row m, columns 8*kg..) at byte (m / rb * kb + kg / 8) * rb * 256 + (kg % 8) * rb * 32 +
+  // (m % rb / 8) * 128 + (m % 8) * 16, low parts rb * 16 bytes further)
+  unsigned char* img;
+  int img_rb, img_kb;
 };
+
+__device__ __forceinline__ void attn_store(const AttnParams& ap, float* dst, int m, int col, float v) {
+  if (ap.img == nullptr) {
+    dst[col] = v;
+    return;
+  }
+  const int rb = m / ap.img_rb, tm = m - rb * ap.img_rb, kg = col >> 3;
+  unsigned char* p = ap.img + ((size_t)rb * ap.img_kb + (kg >> 3)) * ((size_t)ap.img_rb * 256) + (size_t)(kg & 7) * (ap.img_rb * 32) +
+                     (size_t)(tm >> 3) * 128 + (tm & 7) * 16 + (col & 7) * 2;
+  const __nv_bfloat16 hi = __float2bfloat16_rn(v);
+  *reinterpret_cast<__nv_bfloat16*>(p) = hi;
+  *reinterpret_cast<__nv_bfloat16*>(p + (size_t)ap.img_rb * 16) = __float2bfloat16_rn(v - __bfloat162float(hi));
+}
 
 template <typename KT, int HD>
 __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnParams ap) {
@@ -170,9 +189,9 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnParams ap) 
   if (tid == 0) ap.counters[b * ap.n_heads + head] = 0;
   for (int i = 0; i < R; ++i) {
     const int pos = s_pos[i];
-    float* dst = ap.out + (size_t)(row0 + i) * d_model + head * HD;
+    float* dst = ap.out + (size_t)(row0 + i) * d_model;
     if (pos < 0) {
-      for (int d = tid; d < HD; d += kAttnThreads) dst[d] = 0.f;
+      for (int d = tid; d < HD; d += kAttnThreads) attn_store(ap, dst, row0 + i, head * HD + d, 0.f);
       continue;
     }
     const int nc = pos / C + 1;
@@ -187,7 +206,7 @@ __global__ void __launch_bounds__(kAttnThreads) attention_kernel(AttnParams ap) 
       float o = 0.f;
       for (int cc = 0; cc < nc; ++cc)
         o = fmaf(__ldcg(po + (size_t)cc * HD + d), __expf(__ldcg(ml + cc * 2) - mx), o);
-      dst[d] = o * inv_l;
+      attn_store(ap, dst, row0 + i, head * HD + d, o * inv_l);
     }
   }
 }

@@ -112,6 +112,9 @@ struct sdfp_ctx {
   bool dense_decode = false;       // ... this context's decode passes run on it as well
   void* um_lm_head = nullptr;
   unsigned char* um_x = nullptr;   // activation image, rows_cap (rounded to 128) x widest K
+  // decode on the dense path: images of gain * h, of the attention output and of u; sums of squares
+  unsigned char *um_xh = nullptr, *um_xa = nullptr, *um_xu = nullptr;
+  float* um_ssq = nullptr;
   float* um_partial = nullptr;
   int *um_flags = nullptr, *um_error = nullptr;
   int rows_cap = kMaxRows;         // rows the activation buffers h, q, att, u and the row plan hold
@@ -188,19 +191,11 @@ int linear_grid_fma(const sdfp_ctx* c, int n_pairs) {
   return std::max(1, std::min(want, c->num_sms * 8));
 }
 
-// Linear layer on the tcgen05 path: activation image (RMSNorm folded in), then the stream-K kernel.
-// Launched in plain stream order (no programmatic dependent launch): the kernel holds all of an
-// SM's tensor memory and nearly all of its shared memory, so nothing should share the SM with it.
-cudaError_t run_dense_linear(sdfp_ctx* c, const void* w_img, const float* x, int ldx, int rows, int K, int n_pairs,
-                             const float* gain, const EpiParams& ep) {
-  const int RB = rows >= kUmMaxRB ? kUmMaxRB : ((rows + 15) / 16) * 16;
-  const int KB = (K + kUmBK - 1) / kUmBK;
-  cudaError_t e = launch(c, prep_rows_kernel, dim3((rows + 7) / 8), dim3(kPrepThreads), 0, x, ldx, rows, K, gain, c->cfg.rms_eps,
-                         c->um_x, RB, KB);
-  if (e != cudaSuccess) return e;
+UmmaParams dense_params(const sdfp_ctx* c, const void* w_img, const unsigned char* x_img, int rows, int RB, int KB, int n_pairs,
+                        const EpiParams& ep) {
   UmmaParams p{};
   p.W = reinterpret_cast<const unsigned char*>(w_img);
-  p.X = c->um_x;
+  p.X = x_img;
   p.n_ft = (n_pairs + 63) / 64;
   p.n_rb = (rows + RB - 1) / RB;
   p.KB = KB;
@@ -211,10 +206,31 @@ cudaError_t run_dense_linear(sdfp_ctx* c, const void* w_img, const float* x, int
   p.partial = c->um_partial;
   p.flags = c->um_flags;
   p.error = c->um_error;
+  p.ssq_ld = kMaxRows;
+  p.inv_k = 1.0f;
+  p.eps = c->cfg.rms_eps;
   p.ep = ep;
-  c->launches += 1;
-  umma_linear_kernel<<<c->num_sms, kUmThreads, umma_smem_bytes(RB, p.n_stages), c->stream>>>(p);
-  return cudaGetLastError();
+  return p;
+}
+
+// One CTA per SM.  Launched with the programmatic-dependent-launch attribute like every other
+// kernel: the kernel requests its first weights before it waits for its predecessor.
+cudaError_t launch_dense(sdfp_ctx* c, const UmmaParams& p) {
+  return launch(c, umma_linear_kernel, dim3(c->num_sms), dim3(kUmThreads), umma_smem_bytes(p.RB, p.n_stages), p);
+}
+
+// Linear layer on the tcgen05 path from fp32 rows: activation image (RMSNorm folded in) by a
+// conversion kernel, then the stream-K kernel.  (The prompt pass; decode passes on the dense path
+// chain the kernels image to image instead, see enqueue_dense_pass.)
+cudaError_t run_dense_linear(sdfp_ctx* c, const void* w_img, const float* x, int ldx, int rows, int K, int n_pairs,
+                             const float* gain, const EpiParams& ep) {
+  const int RB = rows >= kUmMaxRB ? kUmMaxRB : ((rows + 15) / 16) * 16;
+  const int KB = (K + kUmBK - 1) / kUmBK;
+  cudaError_t e = launch(c, prep_rows_kernel, dim3((rows + 7) / 8), dim3(kPrepThreads), 0, x, ldx, rows, K, gain, c->cfg.rms_eps,
+                         c->um_x, RB, KB);
+  if (e != cudaSuccess) return e;
+  const UmmaParams p = dense_params(c, w_img, c->um_x, rows, RB, KB, n_pairs, ep);
+  return launch_dense(c, p);
 }
 
 cudaError_t run_linear(sdfp_ctx* c, const LinearCall& lc) {
@@ -252,8 +268,12 @@ cudaError_t launch_attention_t(sdfp_ctx* c, const AttnParams& ap, int n_groups) 
   return launch(c, attention_kernel<KT, HD>, dim3(ap.n_chunks, ap.n_heads, n_groups), dim3(kAttnThreads), smem, ap);
 }
 
-cudaError_t run_attention(sdfp_ctx* c, const KvCache& kv, int layer, int rows, int rows_per_seq, int n_chunks) {
+cudaError_t run_attention(sdfp_ctx* c, const KvCache& kv, int layer, int rows, int rows_per_seq, int n_chunks,
+                          unsigned char* img = nullptr, int img_rb = 0, int img_kb = 0) {
   AttnParams ap{};
+  ap.img = img;
+  ap.img_rb = img_rb;
+  ap.img_kb = img_kb;
   ap.q = c->q;
   ap.kcache = kv.k[layer];
   ap.vcache = kv.v[layer];
@@ -462,6 +482,8 @@ cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool w
 // prompts shorter than this go through the decode kernels in chunks (a handful of launches)
 constexpr int kDenseMinRows = 16;
 
+int enqueue_dense_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn_rows_per_seq, int n_chunks, int decide);
+
 enum Decide { DECIDE_NONE = 0, DECIDE_LOGITS = 1, DECIDE_ARGMAX = 2, DECIDE_SAMPLE_DRAFT = 3 };
 
 // rows: total rows; rows_per_seq for the attention grouping; n_chunks bounds the context.
@@ -469,14 +491,15 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
                  int decide) {
   const sdfp_config& g = c->cfg;
   const int d = g.d_model, f = g.d_ffn;
+  if (c->dense_decode) return enqueue_dense_pass(c, pd, draft, rows, attn_rows_per_seq, n_chunks, decide);
   if (c->bf16)
     CU_OK(c, launch(c, plan_embed_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs,
                     (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
-                    reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, d));
+                    reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, d, EmbedImage{}));
   else
     CU_OK(c, launch(c, plan_embed_kernel<float>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs,
                     (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
-                    reinterpret_cast<const float*>(c->embed), c->h, d));
+                    reinterpret_cast<const float*>(c->embed), c->h, d, EmbedImage{}));
   const KvCache& kv = draft ? c->cache_d : c->cache_t;
   const bool whole_pass = c->use_pass;  // a context takes ONE path for all its passes (see sdfp_create)
   if (whole_pass && rows > kPassMaxRows) return fail(c, SDFP_ESTATE, "a pass of %d rows reached the whole-pass kernel", rows);
@@ -512,6 +535,86 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
   if (decide == DECIDE_ARGMAX)
     CU_OK(c, launch(c, argmax_kernel, dim3(rows), dim3(kArgmaxThreads), 0, (const float*)c->logits, g.vocab, pd,
                     c->draft_tok, c->tgt_tok, c->row_argmax));
+  else if (decide == DECIDE_SAMPLE_DRAFT)
+    CU_OK(c, launch(c, sample_draft_kernel, dim3(rows), dim3(kSampleThreads), 0, (const float*)c->logits, g.vocab, pd,
+                    (const GenState*)c->gs, c->draft_tok, c->qprob, c->qsum));
+  return 0;
+}
+
+// One forward pass of a context that decodes on the dense path: every linear layer is one launch of
+// the tcgen05 kernel, and the kernels hand the activations on as operand images: the embedding
+// kernel and the epilogues that write the residual stream leave (next norm's gain) * h as bf16
+// hi + lo plus partial sums of squares, the next linear layer applies 1/rms to its accumulators;
+// the SwiGLU epilogue leaves the image of u, the attention kernel the image of its output.
+int enqueue_dense_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn_rows_per_seq, int n_chunks, int decide) {
+  const sdfp_config& g = c->cfg;
+  const int d = g.d_model, f = g.d_ffn;
+  const int RB = ((rows + 15) / 16) * 16;
+  const int KBd = (d + kUmBK - 1) / kUmBK, KBf = (f + kUmBK - 1) / kUmBK;
+  const KvCache& kv = draft ? c->cache_d : c->cache_t;
+  struct Block {
+    int layer;
+    bool attn;
+  };
+  std::vector<Block> blocks;
+  for (int l = 0; l < g.n_layers; ++l) {
+    if (!draft || c->keep_attn[l]) blocks.push_back({l, true});
+    if (!draft || c->keep_ffn[l]) blocks.push_back({l, false});
+  }
+  auto gain_of = [&](size_t i) -> const float* {  // the gain of the norm in front of block i (the final norm behind the last)
+    if (i >= blocks.size()) return c->final_gain;
+    const LayerWeights& lw = c->layers[blocks[i].layer];
+    return blocks[i].attn ? lw.attn_gain : lw.ffn_gain;
+  };
+  CU_OK(c, launch(c, plan_embed_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs, (const int*)c->seq_tok,
+                  g.max_seq, (const int*)c->draft_tok, c->plan, reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, d,
+                  EmbedImage{c->um_xh, gain_of(0), c->um_ssq, RB, KBd}));
+  int groups = 1;  // partial sums of squares per row the next norm has to add
+  const int resid_tiles = (d / 2 + 63) / 64;
+  auto normed = [&](UmmaParams& p) {
+    p.ssq_in = c->um_ssq;
+    p.ssq_groups = groups;
+    p.inv_k = 1.0f / (float)d;
+  };
+  auto resid_out = [&](UmmaParams& p, size_t next_block) {
+    p.img_out = c->um_xh;
+    p.img_KB = KBd;
+    p.gain_out = gain_of(next_block);
+    p.ssq_out = c->um_ssq;
+  };
+  for (size_t i = 0; i < blocks.size(); ++i) {
+    const int l = blocks[i].layer;
+    const LayerWeights& lw = c->layers[l];
+    if (blocks[i].attn) {
+      EpiParams qkv = base_epi(c, EPI_QKV, c->q, d);
+      qkv.kcache = kv.k[l];
+      qkv.vcache = kv.v[l];
+      UmmaParams p = dense_params(c, lw.um_qkv, c->um_xh, rows, RB, KBd, 3 * d / 2, qkv);
+      normed(p);
+      CU_OK(c, launch_dense(c, p));
+      CU_OK(c, run_attention(c, kv, l, rows, attn_rows_per_seq, n_chunks, c->um_xa, RB, KBd));
+      UmmaParams o = dense_params(c, lw.um_wo, c->um_xa, rows, RB, KBd, d / 2, base_epi(c, EPI_RESID, c->h, d));
+      resid_out(o, i + 1);
+      CU_OK(c, launch_dense(c, o));
+    } else {
+      UmmaParams p = dense_params(c, lw.um_gu, c->um_xh, rows, RB, KBd, f, base_epi(c, EPI_SWIGLU, nullptr, f));
+      normed(p);
+      p.img_out = c->um_xu;
+      p.img_KB = KBf;
+      CU_OK(c, launch_dense(c, p));
+      UmmaParams dn = dense_params(c, lw.um_down, c->um_xu, rows, RB, KBf, d / 2, base_epi(c, EPI_RESID, c->h, d));
+      resid_out(dn, i + 1);
+      CU_OK(c, launch_dense(c, dn));
+    }
+    groups = resid_tiles;
+  }
+  if (decide == DECIDE_NONE) return 0;
+  UmmaParams lm = dense_params(c, c->um_lm_head, c->um_xh, rows, RB, KBd, g.vocab / 2, base_epi(c, EPI_LOGITS, c->logits, g.vocab));
+  normed(lm);
+  CU_OK(c, launch_dense(c, lm));
+  if (decide == DECIDE_ARGMAX)
+    CU_OK(c, launch(c, argmax_kernel, dim3(rows), dim3(kArgmaxThreads), 0, (const float*)c->logits, g.vocab, pd, c->draft_tok,
+                    c->tgt_tok, c->row_argmax));
   else if (decide == DECIDE_SAMPLE_DRAFT)
     CU_OK(c, launch(c, sample_draft_kernel, dim3(rows), dim3(kSampleThreads), 0, (const float*)c->logits, g.vocab, pd,
                     (const GenState*)c->gs, c->draft_tok, c->qprob, c->qsum));
@@ -827,6 +930,13 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
         (r = dev_alloc(c, &c->um_flags, (size_t)c->num_sms, true)) || (r = dev_alloc(c, &c->um_error, 1, true)) ||
         (r = dev_alloc(c, &c->h_fork, R * g.d_model)))
       return bail(r);
+    if (c->dense_decode) {
+      const size_t kd = (size_t)(((g.d_model + kUmBK - 1) / kUmBK) * kUmBK), kf = (size_t)(((g.d_ffn + kUmBK - 1) / kUmBK) * kUmBK);
+      if ((r = dev_alloc(c, &c->um_xh, (size_t)kMaxRows * kd * 4, true)) || (r = dev_alloc(c, &c->um_xa, (size_t)kMaxRows * kd * 4, true)) ||
+          (r = dev_alloc(c, &c->um_xu, (size_t)kMaxRows * kf * 4, true)) ||
+          (r = dev_alloc(c, &c->um_ssq, (size_t)kSsqMaxGroups * kMaxRows, true)))
+        return bail(r);
+    }
   }
   if (c->use_pass) {
     if ((r = dev_alloc(c, &c->psync, 1, true)) ||
@@ -1024,7 +1134,7 @@ int prefill_dense(sdfp_ctx* c, int b, int rows_t, int rows_d, bool with_draft) {
   pd.count = rows_t;
   pd.src = c->seq_tok + (size_t)b * g.max_seq;
   CU_OK(c, launch(c, plan_embed_kernel<__nv_bfloat16>, dim3(rows_t), dim3(128), 0, pd, (const GenState*)c->gs, (const int*)c->seq_tok,
-                  g.max_seq, (const int*)c->draft_tok, c->plan, reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, d));
+                  g.max_seq, (const int*)c->draft_tok, c->plan, reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, d, EmbedImage{}));
   const int fork = with_draft ? first_pruned_layer(c) : -1;  // the draft's residual rows leave the target's after this many layers
   const size_t fork_bytes = (size_t)rows_d * d * sizeof(float);
   if (fork == 0 && rows_d > 0) CU_OK(c, cudaMemcpyAsync(c->h_fork, c->h, fork_bytes, cudaMemcpyDeviceToDevice, c->stream));
@@ -1331,7 +1441,7 @@ extern "C" int sdfp_time_pass(sdfp_ctx* c, int32_t draft, int32_t rows, int32_t 
   auto plan = [&]() -> cudaError_t {
     return launch(c, plan_embed_kernel<__nv_bfloat16>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs,
                   (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
-                  reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, g.d_model);
+                  reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, g.d_model, EmbedImage{});
   };
   for (int i = 0; i < 3 && err == cudaSuccess; ++i) {  // warm-up
     err = plan();
@@ -1374,8 +1484,27 @@ extern "C" int sdfp_time_linear(sdfp_ctx* c, int32_t which, int32_t rows, int32_
   // rows carry nothing (position -1): the QKV epilogue then writes no cache entry
   CU_OK(c, cudaMemsetAsync(c->plan.row_pos, 0xff, kMaxRows * 4, c->stream));
   CU_OK(c, cudaMemsetAsync(c->plan.row_seq, 0, kMaxRows * 4, c->stream));
+  // contexts that decode on the dense path: the activation image is made once, outside the timed
+  // launches (in a pass the preceding kernel's epilogue leaves it), and one launch = one tcgen05 kernel
+  const bool dense = c->dense_decode;
+  const int RB = ((rows + 15) / 16) * 16;
+  const int Kin = which == 3 ? f : d, KBin = (Kin + kUmBK - 1) / kUmBK;
+  if (dense)
+    CU_OK(c, launch(c, prep_rows_kernel, dim3((rows + 7) / 8), dim3(kPrepThreads), 0, (const float*)(which == 3 ? c->u : c->h),
+                    Kin, (int)rows, Kin, (const float*)nullptr, g.rms_eps, c->um_x, RB, KBin));
   auto one = [&](int l) -> cudaError_t {
     const LayerWeights& lw = c->layers[l % g.n_layers];
+    if (dense) {
+      const void* w = which == 0 ? lw.um_qkv : which == 1 ? lw.um_wo : which == 2 ? lw.um_gu : which == 3 ? lw.um_down : c->um_lm_head;
+      const int n_pairs = which == 0 ? 3 * d / 2 : which == 2 ? f : which == 4 ? g.vocab / 2 : d / 2;
+      EpiParams ep = which == 0 ? base_epi(c, EPI_QKV, c->q, d)
+                     : which == 2 ? base_epi(c, EPI_SWIGLU, c->u, f)
+                     : which == 4 ? base_epi(c, EPI_LOGITS, c->logits, g.vocab)
+                                  : base_epi(c, EPI_RESID, c->q, d);
+      ep.kcache = c->cache_t.k[0];
+      ep.vcache = c->cache_t.v[0];
+      return launch_dense(c, dense_params(c, w, c->um_x, rows, RB, KBin, n_pairs, ep));
+    }
     if (which == 0) {
       LinearCall lc{lw.qkv, c->h, d, rows, d, 3 * d / 2, lw.attn_gain, base_epi(c, EPI_QKV, c->q, d)};
       lc.ep.kcache = c->cache_t.k[0];

@@ -42,14 +42,24 @@ struct RowPlan {
   int* row_tok;
 };
 
+// Dense path: the embedding rows also go out as the activation image of the first linear layer
+// (gain * h as bf16 hi + lo, layout of umma_linear.cuh) together with each row's sum of squares.
+struct EmbedImage {
+  unsigned char* img;  // null: none
+  const float* gain;
+  float* ssq;          // [rows]
+  int rb, kb;
+};
+
 // One CTA per row: decide which token sits in the row and where, then gather its
 // embedding into the residual stream h[row, :].
 template <typename WT>
 __global__ void __launch_bounds__(128)
 plan_embed_kernel(PassDesc pd, const GenState* gs, const int* seq_tok, int max_seq,
                   const int* draft_tok, RowPlan plan, const WT* __restrict__ embed, float* __restrict__ h,
-                  int d_model) {
+                  int d_model, EmbedImage im) {
   __shared__ int s_tok, s_pos;
+  __shared__ float s_sq[128];
   pdl_wait();
   pdl_launch_dependents();
   const int m = blockIdx.x;
@@ -88,10 +98,41 @@ plan_embed_kernel(PassDesc pd, const GenState* gs, const int* seq_tok, int max_s
   __syncthreads();
   const WT* e = embed + (size_t)s_tok * d_model;
   float* dst = h + (size_t)m * d_model;
+  float sq = 0.f;
   for (int k = threadIdx.x * 4; k < d_model; k += blockDim.x * 4) {
     float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
     if (s_pos >= 0) v = load4(e + k);
     *reinterpret_cast<float4*>(dst + k) = v;
+    if (im.img != nullptr) {
+      sq = fmaf(v.x, v.x, sq);
+      sq = fmaf(v.y, v.y, sq);
+      sq = fmaf(v.z, v.z, sq);
+      sq = fmaf(v.w, v.w, sq);
+      const float4 g = *reinterpret_cast<const float4*>(im.gain + k);
+      const float x0 = v.x * g.x, x1 = v.y * g.y, x2 = v.z * g.z, x3 = v.w * g.w;
+      const __nv_bfloat16 h0 = __float2bfloat16_rn(x0), h1 = __float2bfloat16_rn(x1), h2 = __float2bfloat16_rn(x2), h3 = __float2bfloat16_rn(x3);
+      const __nv_bfloat16 l0 = __float2bfloat16_rn(x0 - __bfloat162float(h0)), l1 = __float2bfloat16_rn(x1 - __bfloat162float(h1));
+      const __nv_bfloat16 l2 = __float2bfloat16_rn(x2 - __bfloat162float(h2)), l3 = __float2bfloat16_rn(x3 - __bfloat162float(h3));
+      const int rb = m / im.rb, tm = m - rb * im.rb, kg = k >> 3;
+      unsigned char* p = im.img + ((size_t)rb * im.kb + (kg >> 3)) * ((size_t)im.rb * 256) + (size_t)(kg & 7) * (im.rb * 32) +
+                         (size_t)(tm >> 3) * 128 + (tm & 7) * 16 + (k & 7) * 2;
+      uint2 hv, lv;
+      hv.x = (uint32_t)__bfloat16_as_ushort(h0) | ((uint32_t)__bfloat16_as_ushort(h1) << 16);
+      hv.y = (uint32_t)__bfloat16_as_ushort(h2) | ((uint32_t)__bfloat16_as_ushort(h3) << 16);
+      lv.x = (uint32_t)__bfloat16_as_ushort(l0) | ((uint32_t)__bfloat16_as_ushort(l1) << 16);
+      lv.y = (uint32_t)__bfloat16_as_ushort(l2) | ((uint32_t)__bfloat16_as_ushort(l3) << 16);
+      *reinterpret_cast<uint2*>(p) = hv;
+      *reinterpret_cast<uint2*>(p + (size_t)im.rb * 16) = lv;
+    }
+  }
+  if (im.img != nullptr) {  // the row's sum of squares, thread partials added in thread order
+    s_sq[threadIdx.x] = sq;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+      float t = 0.f;
+      for (int i = 0; i < (int)blockDim.x; ++i) t += s_sq[i];
+      im.ssq[m] = t;
+    }
   }
 }
 

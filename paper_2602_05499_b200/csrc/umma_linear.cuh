@@ -66,6 +66,7 @@ struct UmmaShared {
   int decision;  // abort as sampled by one epilogue thread between two barriers
   int n_posts;
   int posts[160];
+  float inv[kUmMaxRB];  // 1/rms of the rows of the running tile
 };
 
 inline size_t umma_smem_bytes(int RB, int n_stages) {
@@ -87,8 +88,30 @@ struct UmmaParams {
   float* partial;          // [grid][RB * 128] partial accumulators of cut tiles
   int* flags;              // [grid], zero between launches
   int* error;              // first UmmaError seen, sticky
+  // RMSNorm folded in: the activation image carries gain * h; 1/rms of row m comes from ssq_groups
+  // partial sums of squares ssq_in[g * ssq_ld + m] left by whoever wrote h (null: no norm)
+  const float* ssq_in;
+  int ssq_groups, ssq_ld;
+  float inv_k, eps;
+  // The epilogue can leave its result as the activation image of the NEXT linear layer (row block
+  // size RB, k blocks img_KB), so that no conversion kernel runs between the two:
+  //   EPI_SWIGLU  image of u (img_out non-null); the fp32 copy is written only if ep.out is non-null
+  //   EPI_RESID   image of gain_out * h_new, and this tile's sum of squares of h_new per row in
+  //               ssq_out[tile * ssq_ld + m]
+  unsigned char* img_out;
+  int img_KB;
+  const float* gain_out;
+  float* ssq_out;
   EpiParams ep;
 };
+
+// byte offset of the 16-byte piece (row m, k group kg = k / 8) of the high parts in an activation image
+__host__ __device__ __forceinline__ size_t um_img_offset(int RB, int KB, int m, int kg) {
+  const int rb = m / RB, tm = m - rb * RB;
+  return ((size_t)rb * KB + (kg >> 3)) * (size_t)um_b_stage_bytes(RB) + (size_t)(kg & 7) * (RB * 32) + (size_t)(tm >> 3) * 128 + (tm & 7) * 16;
+}
+// ... and from there to the piece of the low parts
+__host__ __device__ __forceinline__ size_t um_img_lo(int RB) { return (size_t)(RB / 8) * 128; }
 
 // ---- tcgen05 / descriptor helpers ----------------------------------------------------------------
 // Shared-memory matrix descriptor, K-major, no swizzle: start address, leading-dimension byte offset
@@ -196,6 +219,10 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
   um_fence_after();
   const uint32_t tmem_base = sh->tmem_base;
   volatile int* s_abort = &sh->abort;
+  // The next kernel of the stream may be scheduled from here on: its CTAs find room only where a
+  // CTA of this kernel has exited (shared memory), and they wait for this whole grid before they
+  // touch anything it writes.
+  pdl_launch_dependents();
 
   auto next_seg = [&](long long u) {
     UmSeg s;
@@ -215,27 +242,47 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
       int stage = 0;
       unsigned phase = 0, issued = 0;
       bool ok = true;
-      for (long long u = ub; u < ue && ok;) {
-        const UmSeg s = next_seg(u);
-        const int ft = s.tile / p.n_rb, rb = s.tile - ft * p.n_rb;
-        const unsigned char* wsrc = p.W + ((size_t)ft * KB + s.kb0) * kUmABytes;
-        const unsigned char* xsrc = p.X + ((size_t)rb * KB + s.kb0) * um_b_stage_bytes(p.RB);
-        for (int kb = s.kb0; kb < s.kb1; ++kb) {
-          ok = um_wait([&] { return mbar_try_wait(&sh->empty[stage], phase ^ 1u); }, p.error, s_abort, UMMA_ERR_STAGE_EMPTY);
-          if (!ok) break;
-          unsigned char* dst = smem + (size_t)stage * stage_bytes;
-          mbar_arrive_expect_tx(&sh->full[stage], (unsigned)stage_bytes);
-          bulk_load(dst, wsrc, kUmABytes, &sh->full[stage], pol);
-          bulk_load(dst + kUmABytes, xsrc, (unsigned)um_b_stage_bytes(p.RB), &sh->full[stage], pol_x);
-          wsrc += kUmABytes;
-          xsrc += um_b_stage_bytes(p.RB);
-          ++issued;
-          if (++stage == p.n_stages) {
-            stage = 0;
-            phase ^= 1u;
+      // Weights do not depend on the kernels before this one: the first ring's worth of weight
+      // blocks is requested before the wait on the preceding kernel, the activation blocks of the
+      // same stages right after it.
+      for (int pass = 0; pass < 2 && ok; ++pass) {
+        unsigned i = 0;  // k blocks of this CTA in order
+        stage = 0;
+        phase = 0;
+        for (long long u = ub; u < ue && ok;) {
+          const UmSeg s = next_seg(u);
+          const int ft = s.tile / p.n_rb, rb = s.tile - ft * p.n_rb;
+          const unsigned char* wsrc = p.W + ((size_t)ft * KB + s.kb0) * kUmABytes;
+          const unsigned char* xsrc = p.X + ((size_t)rb * KB + s.kb0) * um_b_stage_bytes(p.RB);
+          for (int kb = s.kb0; kb < s.kb1; ++kb, ++i) {
+            const bool early = i < (unsigned)p.n_stages;  // first use of its stage: nothing to wait for
+            if (pass == 0 && !early) break;
+            unsigned char* dst = smem + (size_t)stage * stage_bytes;
+            if (pass == 0) {
+              mbar_arrive_expect_tx(&sh->full[stage], (unsigned)stage_bytes);
+              bulk_load(dst, wsrc, kUmABytes, &sh->full[stage], pol);
+              ++issued;
+            } else if (early) {
+              bulk_load(dst + kUmABytes, xsrc, (unsigned)um_b_stage_bytes(p.RB), &sh->full[stage], pol_x);
+            } else {
+              ok = um_wait([&] { return mbar_try_wait(&sh->empty[stage], phase ^ 1u); }, p.error, s_abort, UMMA_ERR_STAGE_EMPTY);
+              if (!ok) break;
+              mbar_arrive_expect_tx(&sh->full[stage], (unsigned)stage_bytes);
+              bulk_load(dst, wsrc, kUmABytes, &sh->full[stage], pol);
+              bulk_load(dst + kUmABytes, xsrc, (unsigned)um_b_stage_bytes(p.RB), &sh->full[stage], pol_x);
+              ++issued;
+            }
+            wsrc += kUmABytes;
+            xsrc += um_b_stage_bytes(p.RB);
+            if (++stage == p.n_stages) {
+              stage = 0;
+              phase ^= 1u;
+            }
           }
+          if (pass == 0 && i >= (unsigned)p.n_stages) break;
+          u += s.kb1 - s.kb0;
         }
-        u += s.kb1 - s.kb0;
+        if (pass == 0) pdl_wait();  // the activation image is the preceding kernel's output
       }
       if (!ok) {
         // nothing may still be landing in shared memory when the CTA exits
@@ -295,6 +342,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
     int buf = 0;
     unsigned acc_phase = 0;
     const int RB = p.RB;
+    pdl_wait();  // everything this role reads or writes in global memory belongs to the stream's order
     for (long long u = ub; u < ue;) {
       const UmSeg s = next_seg(u);
       const int ft = s.tile / p.n_rb, rb = s.tile - ft * p.n_rb;
@@ -324,6 +372,16 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
       um_fence_after();
       const int n_posts = owner ? sh->n_posts : 0;
       const int row0 = rb * RB;
+      if (starts && p.ssq_in != nullptr) {
+        // 1/rms of this tile's rows: the partial sums are asked for together and added in group order
+        if (et < RB && row0 + et < p.M) {
+          float ssum = 0.f;
+#pragma unroll 8
+          for (int g2 = 0; g2 < p.ssq_groups; ++g2) ssum += __ldcg(p.ssq_in + (size_t)g2 * p.ssq_ld + row0 + et);
+          sh->inv[et] = rsqrtf(ssum * p.inv_k + p.eps);
+        }
+        um_epi_sync();
+      }
       float* my_post = p.partial + (size_t)cta * (RB * kUmFeat);
       for (int c = 0; c < RB / kUmChunk; ++c) {
         if (row0 + c * kUmChunk >= p.M) break;  // rows that carry nothing (uniform)
@@ -348,14 +406,82 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
         for (int t = 0; t < 16; ++t) ex[R * kUmExLd + t] = hi[t];
         um_epi_sync();
         const int pg = ft * 64 + pl;
+        const bool want_img = p.img_out != nullptr;
+        float keep0[8], keep1[8];  // results this thread owes the output image
 #pragma unroll
         for (int t8 = 0; t8 < 8; ++t8) {
           const int t = half * 8 + t8;
           const int m = row0 + c * kUmChunk + t;
-          const float v0 = ex[pl * kUmExLd + t], v1 = ex[(pl + 64) * kUmExLd + t];
-          if (m < p.M && pg < p.n_pairs) apply_epilogue<__nv_bfloat16>(p.ep, pg, m, v0, v1);
+          float v0 = ex[pl * kUmExLd + t], v1 = ex[(pl + 64) * kUmExLd + t];
+          keep0[t8] = 0.f;
+          keep1[t8] = 0.f;
+          if (m < p.M && pg < p.n_pairs) {
+            if (p.ssq_in != nullptr) {
+              const float inv = sh->inv[c * kUmChunk + t];
+              v0 *= inv;
+              v1 *= inv;
+            }
+            if (p.ep.mode == EPI_RESID && want_img) {
+              const int r0 = ((pg >> 3) << 4) + (pg & 7);
+              float* hp = p.ep.out + (size_t)m * p.ep.out_ld;
+              keep0[t8] = ld_act(hp + r0) + v0;
+              keep1[t8] = ld_act(hp + r0 + 8) + v1;
+              hp[r0] = keep0[t8];
+              hp[r0 + 8] = keep1[t8];
+            } else if (p.ep.mode == EPI_SWIGLU && want_img) {
+              keep0[t8] = (v0 / (1.0f + __expf(-v0))) * v1;
+              if (p.ep.out != nullptr) p.ep.out[(size_t)m * p.ep.out_ld + pg] = keep0[t8];
+            } else {
+              apply_epilogue<__nv_bfloat16>(p.ep, pg, m, v0, v1);
+            }
+          }
         }
-        um_epi_sync();  // ex is rewritten by the next chunk
+        um_epi_sync();  // ex has been read
+        if (want_img) {
+          // results back into ex as [feature of the tile][row], then 16-byte pieces of the image:
+          // 8 consecutive features of one row, high parts and low parts
+          const bool resid = p.ep.mode == EPI_RESID;
+          const int f0 = resid ? ((pl >> 3) << 4) + (pl & 7) : pl;
+#pragma unroll
+          for (int t8 = 0; t8 < 8; ++t8) {
+            ex[f0 * kUmExLd + half * 8 + t8] = keep0[t8];
+            if (resid) ex[(f0 + 8) * kUmExLd + half * 8 + t8] = keep1[t8];
+          }
+          um_epi_sync();
+          const int t = et & 15, m = row0 + c * kUmChunk + t;
+          const int n_kg = resid ? 16 : 8, feat0 = ft * (resid ? 128 : 64);
+          if (m < p.M) {
+            for (int kgl = et >> 4; kgl < n_kg; kgl += 8) {
+              float v[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) v[e] = ex[(kgl * 8 + e) * kUmExLd + t];
+              const int k0 = feat0 + kgl * 8;  // first feature of the piece = column of the next layer's input
+              if (k0 >= p.img_KB * kUmBK) continue;
+              if (p.gain_out != nullptr) {
+                const float4 g0 = __ldg(reinterpret_cast<const float4*>(p.gain_out + k0)), g1 = __ldg(reinterpret_cast<const float4*>(p.gain_out + k0 + 4));
+                v[0] *= g0.x; v[1] *= g0.y; v[2] *= g0.z; v[3] *= g0.w;
+                v[4] *= g1.x; v[5] *= g1.y; v[6] *= g1.z; v[7] *= g1.w;
+              }
+              uint4 h4, l4;
+              split_pack(v[0], v[1], h4.x, l4.x);
+              split_pack(v[2], v[3], h4.y, l4.y);
+              split_pack(v[4], v[5], h4.z, l4.z);
+              split_pack(v[6], v[7], h4.w, l4.w);
+              unsigned char* dst = p.img_out + um_img_offset(RB, p.img_KB, m, k0 >> 3);
+              *reinterpret_cast<uint4*>(dst) = h4;
+              *reinterpret_cast<uint4*>(dst + um_img_lo(RB)) = l4;
+            }
+          }
+          if (resid && p.ssq_out != nullptr && et < 16 && row0 + c * kUmChunk + et < p.M) {
+            float ssum = 0.f;  // this tile's 128 features of row et, in feature order
+            for (int fl = 0; fl < kUmFeat; ++fl) {
+              const float x = ex[fl * kUmExLd + et];
+              ssum = fmaf(x, x, ssum);
+            }
+            p.ssq_out[(size_t)ft * p.ssq_ld + row0 + c * kUmChunk + et] = ssum;
+          }
+          um_epi_sync();  // ex is rewritten by the next chunk
+        }
       }
       // tensor memory of this accumulator has been read: hand it back to the MMA warp
       um_fence_before();
