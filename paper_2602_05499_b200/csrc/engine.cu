@@ -23,6 +23,7 @@
 #include "../../include/sdfp.h"
 #include "attention.cuh"
 #include "common.cuh"
+#include "dense_attention.cuh"
 #include "linear_fma.cuh"
 #include "linear_mma.cuh"
 #include "misc_kernels.cuh"
@@ -290,6 +291,21 @@ cudaError_t run_attention(sdfp_ctx* c, const KvCache& kv, int layer, int rows, i
   ap.scale = 1.0f / std::sqrt((float)c->cfg.head_dim);
   const int n_groups = rows / rows_per_seq;
   const bool hd128 = c->cfg.head_dim == 128;
+  if (c->dense_decode) {  // a fixed number of splits per (sequence, head), each walking its chunks
+    const dim3 grid(kAttnSplits, ap.n_heads, n_groups);
+    const dim3 block(kHalfThreads);
+    const int R = rows_per_seq;
+    if (hd128) {
+      const size_t sm = pass_attn_smem_half<128>();
+      if (R <= 2) return launch(c, attention_split_kernel<128, 2>, grid, block, sm, ap, rows);
+      if (R <= 8) return launch(c, attention_split_kernel<128, 8>, grid, block, sm, ap, rows);
+      return launch(c, attention_split_kernel<128, 16>, grid, block, sm, ap, rows);
+    }
+    const size_t sm = pass_attn_smem_half<64>();
+    if (R <= 2) return launch(c, attention_split_kernel<64, 2>, grid, block, sm, ap, rows);
+    if (R <= 8) return launch(c, attention_split_kernel<64, 8>, grid, block, sm, ap, rows);
+    return launch(c, attention_split_kernel<64, 16>, grid, block, sm, ap, rows);
+  }
   if (c->bf16)
     return hd128 ? launch_attention_t<__nv_bfloat16, 128>(c, ap, n_groups)
                  : launch_attention_t<__nv_bfloat16, 64>(c, ap, n_groups);
@@ -904,7 +920,7 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
     }
   }
   const size_t R = (size_t)c->rows_cap;  // prompt rows on the dense path, else the rows of the widest decode pass
-  c->n_chunks_cap = std::max(2, (g.max_seq + kAttnChunk - 1) / kAttnChunk);  // >= 16 rows x kAttnSplits partials
+  c->n_chunks_cap = std::max(kAttnSplits, (g.max_seq + kAttnChunk - 1) / kAttnChunk);  // per (row, head): one partial per 64-key chunk, or kAttnSplits
   c->stats_cap = g.max_seq;
   if ((r = dev_alloc(c, &c->h, R * g.d_model, true)) || (r = dev_alloc(c, &c->q, R * g.d_model, true)) ||
       (r = dev_alloc(c, &c->att, R * g.d_model, true)) || (r = dev_alloc(c, &c->u, R * g.d_ffn, true)) ||
