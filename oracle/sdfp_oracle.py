@@ -48,6 +48,13 @@ design notes of the repository):
       own, and a dropped block is the identity on the residual stream.  `layers` lists
       the layers whose attention block runs, `ffn_layers` those whose FFN block runs
       (None = the same list: whole layers, as in Algorithm 1).
+  R11 KV sharing (Section III-C: the draft is architecture-compatible with the target,
+      "enabling efficient KV reuse during verification"): optionally the draft keeps no
+      cache of its own.  For the committed prefix it attends the TARGET's K/V in the
+      layers it runs; the K/V of the tokens it drafts go into the same cache behind the
+      committed length, where the verification pass overwrites them.  Then no prompt
+      pass of the draft exists and every round's first draft call feeds one token.
+      With a prune set that is a suffix of the stack the two modes coincide exactly.
 
 Pins: see tests/test_oracle_*.py.  The absolute values of the forward pass are
 pinned by an independently written no-cache recomputation, hand-computable
@@ -228,6 +235,16 @@ class CachedLM:
         return _lin(rmsnorm(h, m.w["final_norm"].to(m.dtype), m.rms_eps), m.w["lm_head"])
 
 
+def sharing_draft(target: "CachedLM", layers: Sequence[int], ffn_layers: Optional[Sequence[int]] = None) -> "CachedLM":
+    """A draft model over `target`'s weights that reads and writes the target's cache (R11):
+    the per-layer K/V tensors of the layers it runs ARE the target's tensors."""
+    d = CachedLM(target.m, layers, max_seq=1, ffn_layers=ffn_layers)
+    d.max_seq = target.max_seq
+    d.k = {l: target.k[l] for l in d.layers}
+    d.v = {l: target.v[l] for l in d.layers}
+    return d
+
+
 class StatelessLM:
     """Same interface as CachedLM, but every call recomputes the whole prefix
     with forward_nocache.  `history` must be supplied by the caller through
@@ -345,19 +362,21 @@ def ar_generate(target, prompt: Sequence[int], max_new: int, temperature: float 
 
 def spec_generate(target, draft, prompt: Sequence[int], k: int, max_new: int,
                   temperature: float = 0.0, seed: int = 0, seq: int = 0,
-                  eos_id: int = -1) -> GenResult:
+                  eos_id: int = -1, share_kv: bool = False) -> GenResult:
     """Speculative decoding with a draft that is the target minus some layers.
 
     State between rounds: committed tokens y[0..n−1]; the target's cache holds
     positions 0..n−2; the draft's cache holds 0..n−2 or, after a fully accepted
-    round, 0..n−3 (R8).
+    round, 0..n−3 (R8).  share_kv (R11): `draft` was made by sharing_draft(target, ...);
+    it has no prompt pass and feeds only the last committed token at the start of a round.
     """
     assert k >= 1
     y = [int(t) for t in prompt]
     n0 = len(y)
     if n0 > 1:
         target.feed(y[:-1], 0)
-        draft.feed(y[:-1], 0)
+        if not share_kv:
+            draft.feed(y[:-1], 0)
     draft_cached = n0 - 1            # number of committed positions in the draft cache
     res = GenResult([])
     greedy = (temperature == 0.0)
@@ -415,6 +434,8 @@ def spec_generate(target, draft, prompt: Sequence[int], k: int, max_new: int,
         # (vi) roll back: the target cache is valid through n−1+j = len(y)−2 when
         # nothing was truncated; the draft was fed y[n−1], d_1..d_{k−1}.
         draft_cached = min(n + j, n + k - 1, len(y) - 1)
+        if share_kv:
+            draft_cached = len(y) - 1   # the target's cache holds every committed position but the last
         if eos_id >= 0 and new and new[-1] == eos_id:
             break
     return res

@@ -298,3 +298,28 @@ def test_chi_square_ar_sampling(tiny64):
         cnt[o.categorical(o.softmax_T(logits, T), philox.draw_u(seed, 0, len(prompt), philox.PURPOSE_EXTRA))] += 1
     ob, ex = _merge_small(cnt, p1 * n)
     assert stats.chisquare(ob, ex).pvalue > 1e-3
+
+
+def test_kv_sharing_draft_mode(tiny):
+    """Reading R11.  (a) Greedy output is the target's whatever the draft reads: shared-cache
+    speculative tokens == autoregressive tokens.  (b) A prune set that is a suffix of the stack
+    leaves the draft's K/V equal to the target's in every layer it runs, so the shared-cache run
+    reproduces the separate-cache run exactly, tokens and acceptance counts.  (c) A draft equal to
+    the target accepts everything.  (d) With a prune set in the middle the two modes are
+    different drafts: the acceptance counts differ somewhere."""
+    m, prompt = tiny
+    ar = o.ar_generate(o.CachedLM(m, max_seq=128), prompt, 40).tokens
+
+    def run(kept, share):
+        tgt = o.CachedLM(m, max_seq=128)
+        drf = o.sharing_draft(tgt, kept) if share else o.CachedLM(m, kept, max_seq=128)
+        return o.spec_generate(tgt, drf, prompt, 4, 40, share_kv=share)
+
+    for kept in ([0, 3], [0, 1], [0, 1, 2, 3]):
+        r = run(kept, True)
+        assert r.tokens == ar
+    a, b = run([0, 1], False), run([0, 1], True)
+    assert [x.accepted for x in a.rounds] == [x.accepted for x in b.rounds] and a.tokens == b.tokens
+    assert all(x.accepted == 4 for x in run([0, 1, 2, 3], True).rounds[:-1])
+    a, b = run([0, 3], False), run([0, 3], True)
+    assert [x.accepted for x in a.rounds] != [x.accepted for x in b.rounds]
