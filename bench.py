@@ -212,6 +212,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default="c2-7b-greedy-k4", choices=sorted(WORKLOADS))
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--share-kv", action="store_true", help="the draft attends the target's KV cache (no draft cache, no draft prompt pass)")
     ap.add_argument("--flags", type=int, default=0, help="sdfp_config.flags (1 no graph, 2 no PDL, 4 FMA GEMM, 8 one kernel per operation instead of the whole-pass kernel)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
@@ -241,6 +242,8 @@ def main():
     w = si.make_weights(shape, skip, device=dev, skip_ffn=skip_ffn)
     eng = pkg.Sdfp(shape, w, max_seq=plen + n_new + 16, max_batch=batch, k_max=8, flags=args.flags)
     eng.sdfp_set_draft_sublayers(si.keep_mask(shape.n_layers, skip), si.keep_mask(shape.n_layers, skip_ffn))
+    if args.share_kv:
+        eng.sdfp_set_draft_kv_sharing(True)
     want_cpu = (rank == 0 and world == 1 and not args.no_cpu_baseline)
     w_cpu = si.weights_to(w, "cpu") if want_cpu else None
     del w
@@ -355,7 +358,7 @@ def main():
                        "decoding": "greedy" if temp == 0.0 else "sampled, temperature %g, Philox seed %d" % (temp, SEED),
                        "l2": "inputs larger than L2 (weights %.1f GB per pass)" % (shape.n_params() * 2 / 1e9)
                        if shape.dtype == "bf16" else "tiny model: launch-bound, weights fit in L2",
-                       "replicas": world, "flags": args.flags},
+                       "replicas": world, "flags": args.flags, "draft_shares_target_kv": bool(args.share_kv)},
             "speedup_vs_own_ar": value / world / ar_tok_s,
             "ar_tokens_per_s": ar_tok_s,
             "acceptance_rate": float(np.mean(acc)), "tokens_per_round": float(np.mean(tau)),

@@ -151,6 +151,21 @@ int sdfp_set_draft_layers(sdfp_ctx *ctx, const uint8_t *keep_mask);
 int sdfp_set_draft_sublayers(sdfp_ctx *ctx, const uint8_t *keep_attn, const uint8_t *keep_ffn);
 
 /*
+ * KV reuse between draft and target (Section III-C: the pruned draft stays architecture-
+ * compatible with the target, "enabling efficient KV reuse during verification").  share = 0
+ * (default): the draft has its own cache, filled by its own prompt pass.  share != 0: the draft
+ * keeps no cache; in the layers it runs it attends the TARGET's K/V for the committed prefix and
+ * writes the K/V of the tokens it drafts into the same cache behind the committed length, where
+ * the verification pass overwrites them.  No prompt pass of the draft, no second cache to read,
+ * and each round's first draft pass feeds one token instead of two.  The generated tokens are
+ * the target's either way; the acceptance counts differ unless every pruned block lies behind
+ * every kept one (then both modes are the same computation).  Takes effect at the next
+ * sdfp_generate.  With share != 0 the test hook sdfp_forward_logits(draft = 1) writes the
+ * target's cache.
+ */
+int sdfp_set_draft_kv_sharing(sdfp_ctx *ctx, int32_t share);
+
+/*
  * Generate (Algorithm 1, Stage B).  Synchronous: returns when the outputs are
  * in host memory.
  *   prompts     host int32 [batch, prompt_len], ids in [0, vocab); prompt_len >= 1

@@ -15,7 +15,7 @@ from .build import LIB_PATH
 SDFP_F32, SDFP_BF16 = 0, 1
 FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_FMA_GEMM, FLAG_NO_PASS_KERNEL, FLAG_NO_DENSE = 1, 2, 4, 8, 16
 
-EXPORTS = ["sdfp_create", "sdfp_set_draft_layers", "sdfp_set_draft_sublayers", "sdfp_generate", "sdfp_forward_logits",
+EXPORTS = ["sdfp_create", "sdfp_set_draft_layers", "sdfp_set_draft_sublayers", "sdfp_set_draft_kv_sharing", "sdfp_generate", "sdfp_forward_logits",
            "sdfp_forward_logits_static", "sdfp_get_timing", "sdfp_time_linear", "sdfp_time_pass",
            "sdfp_debug_expire_next_wait", "sdfp_last_error", "sdfp_destroy"]
 
@@ -73,6 +73,8 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdfp_set_draft_layers.restype = C.c_int
     lib.sdfp_set_draft_sublayers.argtypes = [vp, C.POINTER(C.c_uint8), C.POINTER(C.c_uint8)]
     lib.sdfp_set_draft_sublayers.restype = C.c_int
+    lib.sdfp_set_draft_kv_sharing.argtypes = [vp, C.c_int32]
+    lib.sdfp_set_draft_kv_sharing.restype = C.c_int
     lib.sdfp_generate.argtypes = [vp, C.POINTER(C.c_int32), C.c_int32, C.c_int32, C.c_int32, C.c_int32,
                                   C.c_float, C.c_uint64, C.POINTER(C.c_int32), C.POINTER(C.c_int32),
                                   C.POINTER(SdfpRoundStat), C.c_int32, C.POINTER(C.c_int32)]
@@ -186,6 +188,9 @@ class Sdfp:
             raise ValueError("both masks must have n_layers entries")
         self._check(self.lib.sdfp_set_draft_sublayers(self.handle, a.ctypes.data_as(C.POINTER(C.c_uint8)),
                                                       f.ctypes.data_as(C.POINTER(C.c_uint8))))
+
+    def sdfp_set_draft_kv_sharing(self, share: bool):
+        self._check(self.lib.sdfp_set_draft_kv_sharing(self.handle, 1 if share else 0))
 
     def sdfp_generate(self, prompts, k: int, max_new: int, temperature: float = 0.0, seed: int = 0) -> GenOutput:
         p = np.ascontiguousarray(np.asarray(prompts, dtype=np.int32))

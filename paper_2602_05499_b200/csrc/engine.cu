@@ -71,6 +71,7 @@ struct sdfp_ctx {
   float *rope_cos = nullptr, *rope_sin = nullptr;
   KvCache cache_t, cache_d;
   std::vector<uint8_t> keep_attn, keep_ffn;  // draft: which attention blocks and which FFN blocks run
+  bool share_kv = false;  // the draft reads and writes the target's cache instead of its own
 
   // activations / scratch
   float *h = nullptr, *q = nullptr, *att = nullptr, *u = nullptr, *logits = nullptr;
@@ -355,7 +356,7 @@ int build_program(sdfp_ctx* c, bool draft, StageDesc** dev, int* n_out) {
   const sdfp_config& g = c->cfg;
   const int d = g.d_model, f = g.d_ffn;
   const int resid_groups = (d / 16 + kUnitTiles - 1) / kUnitTiles;  // groups of the stages that write the residual stream
-  const KvCache& kv = draft ? c->cache_d : c->cache_t;
+  const KvCache& kv = (draft && !c->share_kv) ? c->cache_d : c->cache_t;
   std::vector<StageDesc> prog;
   for (int l = 0; l < g.n_layers; ++l) {
     const LayerWeights& lw = c->layers[l];
@@ -516,7 +517,7 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
     CU_OK(c, launch(c, plan_embed_kernel<float>, dim3(rows), dim3(128), 0, pd, (const GenState*)c->gs,
                     (const int*)c->seq_tok, g.max_seq, (const int*)c->draft_tok, c->plan,
                     reinterpret_cast<const float*>(c->embed), c->h, d, EmbedImage{}));
-  const KvCache& kv = draft ? c->cache_d : c->cache_t;
+  const KvCache& kv = (draft && !c->share_kv) ? c->cache_d : c->cache_t;
   const bool whole_pass = c->use_pass;  // a context takes ONE path for all its passes (see sdfp_create)
   if (whole_pass && rows > kPassMaxRows) return fail(c, SDFP_ESTATE, "a pass of %d rows reached the whole-pass kernel", rows);
   if (whole_pass) CU_OK(c, run_pass(c, draft, rows, attn_rows_per_seq, decide != DECIDE_NONE));
@@ -567,7 +568,7 @@ int enqueue_dense_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, in
   const int d = g.d_model, f = g.d_ffn;
   const int RB = ((rows + 15) / 16) * 16;
   const int KBd = (d + kUmBK - 1) / kUmBK, KBf = (f + kUmBK - 1) / kUmBK;
-  const KvCache& kv = draft ? c->cache_d : c->cache_t;
+  const KvCache& kv = (draft && !c->share_kv) ? c->cache_d : c->cache_t;
   struct Block {
     int layer;
     bool attn;
@@ -641,9 +642,13 @@ int enqueue_round(sdfp_ctx* c, int k, int batch, bool sampled, int n_chunks) {
   PassDesc pd{};
   pd.n_seq = batch;
   if (k > 0) {
+    // The draft's own cache lags one token after a fully accepted round, so its first pass feeds
+    // the last two committed tokens; a draft that shares the target's cache feeds the last one.
+    const int first_rows = c->share_kv ? 1 : 2;
     pd.kind = PASS_DRAFT_FIRST;
-    pd.rows_per_seq = 2;
-    if (int r = enqueue_pass(c, pd, true, 2 * batch, 2, n_chunks, sampled ? DECIDE_SAMPLE_DRAFT : DECIDE_ARGMAX)) return r;
+    pd.rows_per_seq = first_rows;
+    if (int r = enqueue_pass(c, pd, true, first_rows * batch, first_rows, n_chunks, sampled ? DECIDE_SAMPLE_DRAFT : DECIDE_ARGMAX))
+      return r;
     for (int s = 1; s < k; ++s) {
       pd.kind = PASS_DRAFT_NEXT;
       pd.step = s;
@@ -1002,6 +1007,18 @@ extern "C" int sdfp_set_draft_sublayers(sdfp_ctx* c, const uint8_t* keep_attn, c
   return 0;
 }
 
+extern "C" int sdfp_set_draft_kv_sharing(sdfp_ctx* c, int32_t share) {
+  if (!c) return SDFP_EINVAL;
+  if (int r = check_device(c, "sdfp_set_draft_kv_sharing")) return r;
+  const bool on = share != 0;
+  if (on == c->share_kv) return 0;
+  c->share_kv = on;
+  for (auto& kv : c->graphs) cudaGraphExecDestroy(kv.second.exec);  // captured rounds baked the cache pointers in
+  c->graphs.clear();
+  CU_OK(c, cudaStreamSynchronize(c->stream));
+  return build_programs(c);
+}
+
 extern "C" int sdfp_set_draft_layers(sdfp_ctx* c, const uint8_t* keep_mask) {
   if (!c) return SDFP_EINVAL;
   if (!keep_mask) return fail(c, SDFP_EINVAL, "keep_mask is NULL");
@@ -1222,12 +1239,13 @@ extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch,
   // round always feeds the last two committed tokens)
   CU_OK(c, cudaEventRecord(c->ev[0], st));
   for (int b = 0; b < batch; ++b) {
+    const bool draft_prompt = k > 0 && !c->share_kv;  // a sharing draft has no prompt pass of its own
     if (c->use_dense && prompt_len - 1 >= kDenseMinRows) {
-      if (int r = prefill_dense(c, b, prompt_len - 1, prompt_len - 2, k > 0)) return r;
+      if (int r = prefill_dense(c, b, prompt_len - 1, prompt_len - 2, draft_prompt)) return r;
       continue;
     }
     if (int r = prefill_range(c, false, b, 0, prompt_len - 1)) return r;
-    if (k > 0)
+    if (draft_prompt)
       if (int r = prefill_range(c, true, b, 0, prompt_len - 2)) return r;
   }
   CU_OK(c, cudaEventRecord(c->ev[1], st));
@@ -1317,7 +1335,7 @@ extern "C" int sdfp_generate(sdfp_ctx* c, const int32_t* prompts, int32_t batch,
       if (s.committed == 0 && s.drafted == 0 && k > 0) continue;
       if (k == 0 && s.committed == 0) continue;
       // draft pass i reads keys 0..n-1+i of the kept layers and writes its rows; verify reads 0..n-1+k
-      for (int i = 0; i < k; ++i) t.kv_bytes += (int64_t)kept * kv_tok * ((n[b] + i) + (i == 0 ? 2 : 1));
+      for (int i = 0; i < k; ++i) t.kv_bytes += (int64_t)kept * kv_tok * ((n[b] + i) + (i == 0 && !c->share_kv ? 2 : 1));
       t.kv_bytes += (int64_t)g.n_layers * kv_tok * ((n[b] + k) + (k + 1));
       n[b] += s.committed;
       t.tokens_committed += s.committed;

@@ -25,7 +25,7 @@ struct GenState {
 
 enum PassKind {
   PASS_TOKENS = 0,       // rows r = 0..count-1 of one sequence: token src[r], position start + r
-  PASS_DRAFT_FIRST = 1,  // 2 rows per sequence: the last two committed tokens
+  PASS_DRAFT_FIRST = 1,  // rows_per_seq (2, or 1 when the draft shares the target's cache) rows per sequence: the last committed tokens
   PASS_DRAFT_NEXT = 2,   // 1 row per sequence: draft token number `step` (1-based step >= 1)
   PASS_VERIFY = 3        // k+1 rows per sequence: last committed token, then the k drafts
 };
@@ -78,7 +78,7 @@ plan_embed_kernel(PassDesc pd, const GenState* gs, const int* seq_tok, int max_s
       if (!ld_act(&gs->done[b])) {
         const int n = ld_act(&gs->n[b]);
         if (pd.kind == PASS_DRAFT_FIRST) {
-          pos = n - 2 + i;
+          pos = n - R + i;
           if (pos >= 0) tok = ld_act(seq_tok + (size_t)b * max_seq + pos);
         } else if (pd.kind == PASS_DRAFT_NEXT) {
           pos = n - 1 + pd.step;
@@ -180,7 +180,7 @@ argmax_kernel(const float* logits, int vocab, PassDesc pd, int* draft_tok, int* 
     const int R = pd.rows_per_seq;
     const int b = m / R, i = m - b * R;
     if (pd.kind == PASS_DRAFT_FIRST) {
-      if (i == 1) draft_tok[b * kMaxK + 0] = bi;
+      if (i == R - 1) draft_tok[b * kMaxK + 0] = bi;
     } else if (pd.kind == PASS_DRAFT_NEXT) {
       draft_tok[b * kMaxK + pd.step] = bi;
     } else if (pd.kind == PASS_VERIFY) {

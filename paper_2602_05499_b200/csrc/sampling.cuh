@@ -124,7 +124,7 @@ sample_draft_kernel(const float* logits, int vocab, PassDesc pd, const GenState*
   const int b = m / R, i = m - b * R;
   int s;
   if (pd.kind == PASS_DRAFT_FIRST) {
-    if (i != 1) return;
+    if (i != R - 1) return;
     s = 0;
   } else {
     s = pd.step;

@@ -651,3 +651,64 @@ def test_sublayer_draft_mask(shape, draw, flags):
             eng.sdfp_set_draft_sublayers([0] * shape.n_layers, [0] * shape.n_layers)
     finally:
         eng.close()
+
+
+# ---- the draft sharing the target's KV cache ---------------------------------------------------------
+
+@pytest.mark.parametrize("which", ["f32", "bf16"])
+def test_kv_sharing_draft(tiny, tiny_bf16, which):
+    """sdfp_set_draft_kv_sharing: the draft attends the target's cache for the committed prefix.
+    Tokens stay the target's; acceptance counts follow the oracle's loop in the same mode (fp32:
+    exactly); a suffix prune set gives the same counts in both modes; switching back restores
+    the separate-cache behaviour."""
+    eng, m = tiny if which == "f32" else tiny_bf16
+    prompt = si.make_prompts(m.vocab, 1, 90 if which == "bf16" else 16, seed=90)
+    p = prompt[0].tolist()
+    base = eng.sdfp_generate(prompt, 4, 40)
+    ar = eng.sdfp_generate(prompt, 0, 40)
+    try:
+        eng.sdfp_set_draft_kv_sharing(True)
+        out = eng.sdfp_generate(prompt, 4, 40)
+        assert out.tokens == ar.tokens
+        assert int(out.stats[:, 0, 2].sum()) == 40
+        tgt = orc.CachedLM(m, max_seq=160)
+        ref = orc.spec_generate(tgt, orc.sharing_draft(tgt, [0, 3]), p, 4, 40, share_kv=True)
+        if which == "f32" and ref.tokens == out.tokens[0]:
+            assert out.stats[:, 0, 1].tolist() == [r.accepted for r in ref.rounds]
+        assert out.timing["kv_bytes"] < base.timing["kv_bytes"] or out.n_rounds != base.n_rounds
+        # prune set = the last two layers: the shared cache holds exactly what the draft's own would
+        eng.sdfp_set_draft_layers([1, 1, 0, 0])
+        shared = eng.sdfp_generate(prompt, 4, 40)
+        eng.sdfp_set_draft_kv_sharing(False)
+        own = eng.sdfp_generate(prompt, 4, 40)
+        assert shared.tokens == own.tokens == ar.tokens
+        assert np.array_equal(shared.stats, own.stats)
+    finally:
+        eng.sdfp_set_draft_kv_sharing(False)
+        eng.sdfp_set_draft_layers(si.keep_mask(4, (1, 2)))
+    again = eng.sdfp_generate(prompt, 4, 40)
+    assert again.tokens == base.tokens and np.array_equal(again.stats, base.stats)
+
+
+def test_kv_sharing_draft_batch_and_sampling():
+    """Shared cache with a batch (ragged acceptance) and with sampled decoding against the oracle."""
+    eng, m, _ = make_pair(si.TINY_V64, (1, 2), max_seq=96, max_batch=3, k_max=4)
+    try:
+        eng.sdfp_set_draft_kv_sharing(True)
+        prompts = si.make_prompts(64, 3, 20, seed=91)
+        out = eng.sdfp_generate(prompts, 4, 30)
+        assert out.tokens == eng.sdfp_generate(prompts, 0, 30).tokens
+        for b in range(3):
+            assert eng.sdfp_generate(prompts[b:b + 1], 4, 30).tokens[0] == out.tokens[b]
+        same = 0
+        for seed in range(12):
+            g = eng.sdfp_generate(prompts[:1], 4, 20, temperature=0.125, seed=seed)
+            tgt = orc.CachedLM(m, max_seq=96)
+            ref = orc.spec_generate(tgt, orc.sharing_draft(tgt, [0, 3]), prompts[0].tolist(), 4, 20,
+                                    temperature=0.125, seed=seed, share_kv=True)
+            if g.tokens[0] == ref.tokens:
+                same += 1
+                assert g.stats[:, 0, 1].tolist() == [r.accepted for r in ref.rounds]
+        assert same >= 11
+    finally:
+        eng.close()
