@@ -221,9 +221,10 @@ int sdfp_forward_logits(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int
  *   - SDFP_EINVAL when R x n_heads x P x (head_dim + 2) x 4 bytes, plus the counters, exceed
  *     SDFP_STATIC_SCRATCH_BYTES.  R is the number of rows of the widest pass the call runs and
  *     P the number of partials per (row, head): for bf16 models on the whole-pass kernel
- *     R <= 16 and P = 8, which always fits; with SDFP_FLAG_NO_PASS_KERNEL, with
- *     SDFP_FLAG_FMA_GEMM and for fp32 models R = rows (rounded up to a multiple of 16 beyond
- *     16) and P = ceil((start + rows) / 64).  The message states both sizes.
+ *     R <= 16 and P = 8, which always fits; for bf16 contexts that decode on the dense path
+ *     R = rows (rounded up to a multiple of 16 beyond 16) and P = 8; with
+ *     SDFP_FLAG_NO_PASS_KERNEL, SDFP_FLAG_FMA_GEMM or SDFP_FLAG_NO_DENSE and for fp32 models
+ *     R likewise and P = ceil((start + rows) / 64).  The message states both sizes.
  *   - The first call on a device looks up the array's device address
  *     (cudaGetSymbolAddress, with that device current) and keeps it.  Make that first call
  *     before starting any stream capture, and from one thread: two threads making the first

@@ -587,7 +587,7 @@ int enqueue_dense_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, in
                   g.max_seq, (const int*)c->draft_tok, c->plan, reinterpret_cast<const __nv_bfloat16*>(c->embed), c->h, d,
                   EmbedImage{c->um_xh, gain_of(0), c->um_ssq, RB, KBd}));
   int groups = 1;  // partial sums of squares per row the next norm has to add
-  const int resid_tiles = (d / 2 + 63) / 64;
+  const int resid_tiles = 4 * ((d / 2 + 63) / 64);  // a sum of squares per (32 features, row): four per tile
   auto normed = [&](UmmaParams& p) {
     p.ssq_in = c->um_ssq;
     p.ssq_groups = groups;
@@ -955,7 +955,7 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
       const size_t kd = (size_t)(((g.d_model + kUmBK - 1) / kUmBK) * kUmBK), kf = (size_t)(((g.d_ffn + kUmBK - 1) / kUmBK) * kUmBK);
       if ((r = dev_alloc(c, &c->um_xh, (size_t)kMaxRows * kd * 4, true)) || (r = dev_alloc(c, &c->um_xa, (size_t)kMaxRows * kd * 4, true)) ||
           (r = dev_alloc(c, &c->um_xu, (size_t)kMaxRows * kf * 4, true)) ||
-          (r = dev_alloc(c, &c->um_ssq, (size_t)kSsqMaxGroups * kMaxRows, true)))
+          (r = dev_alloc(c, &c->um_ssq, (size_t)(g.d_model / 32 + 4) * kMaxRows, true)))
         return bail(r);
     }
   }
@@ -1405,7 +1405,7 @@ extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int3
   const int rps = std::min(per_pass, kAttnMaxR);
   const int prow = ((per_pass + rps - 1) / rps) * rps;
   // partials per (row, head): one per 64-key chunk, or a fixed kAttnSplits in the whole-pass kernel
-  const int n_chunks = c->use_pass ? kAttnSplits : (start + rows + kAttnChunk - 1) / kAttnChunk;
+  const int n_chunks = (c->use_pass || c->dense_decode) ? kAttnSplits : (start + rows + kAttnChunk - 1) / kAttnChunk;
   // layout inside the array: arrival counters | (max, sum) partials | o partials
   const size_t counters_bytes = round_up_256((size_t)kMaxRows * g.n_heads * sizeof(int));
   const size_t ml_bytes = round_up_256((size_t)prow * g.n_heads * n_chunks * 2 * sizeof(float));

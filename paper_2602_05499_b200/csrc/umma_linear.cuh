@@ -17,9 +17,10 @@
 // contiguous bytes each), so a pipeline stage is filled by two plain bulk copies:
 //   weights      [feature tile][k block of 64][k group of 8][16 row groups][8 rows][8 elements]
 //   activations  [row block][k block of 64][k group of 8][2*RB/8 row groups][8 rows][8 elements]
-// A k block is four MMA steps (K = 16 each = two k groups).  Inside a feature tile, row r < 64 is
-// the first feature of output pair 64*tile + r and row r + 64 its second (see EpiMode), so the two
-// values a fused epilogue combines (rotary pair, gate/up) sit in lanes r and r + 64.
+// A k block is four MMA steps (K = 16 each = two k groups).  Inside a feature tile, rows 32w..32w+15
+// are the first features of output pairs 64*tile + 16w .. +15 and rows 32w+16..32w+31 their second
+// features (see EpiMode), so the two values a fused epilogue combines (rotary pair, gate/up) sit 16
+// lanes apart in the warp that reads that quarter of tensor memory: one shuffle, no barrier.
 //
 // Work split (stream-K).  Tiles (feature tile, row block) times k blocks form one list of units,
 // cut into equal contiguous ranges, one per CTA (one CTA per SM): every SM streams the same number
@@ -338,11 +339,34 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
     const int et = tid - 64;                 // 0..127
     const int quarter = warp & 3;
     const int R = quarter * 32 + lane;       // tile row (tensor-memory lane) of this thread
-    const int pl = R & 63, half = R >> 6;    // the output pair it finishes and which 8 rows of a chunk
+    const int pl = quarter * 16 + (lane & 15), half = lane >> 4;  // the output pair it finishes and which 8 rows of a chunk
     int buf = 0;
     unsigned acc_phase = 0;
     const int RB = p.RB;
     pdl_wait();  // everything this role reads or writes in global memory belongs to the stream's order
+    // 1/rms of a row block's rows, from the partial sums of squares whoever wrote h left behind:
+    // computed when the role starts (under the MMAs of the first piece) and again only if the row
+    // block changes.  A row's partial sums are asked for 16 at a time and added in group order.
+    int inv_rb = -1;
+    auto ensure_inv = [&](int rb_) {
+      if (p.ssq_in == nullptr || rb_ == inv_rb) return;  // uniform over the role
+      if (inv_rb >= 0) um_epi_sync();                    // the previous block's values are no longer read
+      const int m = rb_ * RB + et;
+      if (et < RB && m < p.M) {
+        float ssum = 0.f;
+        for (int g0 = 0; g0 < p.ssq_groups; g0 += 16) {
+          float part[16];
+#pragma unroll
+          for (int j = 0; j < 16; ++j) part[j] = g0 + j < p.ssq_groups ? __ldcg(p.ssq_in + (size_t)(g0 + j) * p.ssq_ld + m) : 0.f;
+#pragma unroll
+          for (int j = 0; j < 16; ++j) ssum += part[j];
+        }
+        sh->inv[et] = rsqrtf(ssum * p.inv_k + p.eps);
+      }
+      um_epi_sync();
+      inv_rb = rb_;
+    };
+    if (ub < ue) ensure_inv(next_seg(ub).tile % p.n_rb);
     for (long long u = ub; u < ue;) {
       const UmSeg s = next_seg(u);
       const int ft = s.tile / p.n_rb, rb = s.tile - ft * p.n_rb;
@@ -372,16 +396,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
       um_fence_after();
       const int n_posts = owner ? sh->n_posts : 0;
       const int row0 = rb * RB;
-      if (starts && p.ssq_in != nullptr) {
-        // 1/rms of this tile's rows: the partial sums are asked for together and added in group order
-        if (et < RB && row0 + et < p.M) {
-          float ssum = 0.f;
-#pragma unroll 8
-          for (int g2 = 0; g2 < p.ssq_groups; ++g2) ssum += __ldcg(p.ssq_in + (size_t)g2 * p.ssq_ld + row0 + et);
-          sh->inv[et] = rsqrtf(ssum * p.inv_k + p.eps);
-        }
-        um_epi_sync();
-      }
+      ensure_inv(rb);
       float* my_post = p.partial + (size_t)cta * (RB * kUmFeat);
       for (int c = 0; c < RB / kUmChunk; ++c) {
         if (row0 + c * kUmChunk >= p.M) break;  // rows that carry nothing (uniform)
@@ -401,18 +416,18 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
 #pragma unroll
           for (int t = 0; t < 16; ++t) hi[t] += __ldcg(src + t * kUmFeat);
         }
-        // pair exchange: thread (pair pl, half) finishes rows half*8 .. half*8+7 of this chunk
-#pragma unroll
-        for (int t = 0; t < 16; ++t) ex[R * kUmExLd + t] = hi[t];
-        um_epi_sync();
+        // The two features of an output pair sit 16 lanes apart in the same warp: one shuffle per
+        // row brings them together, and thread (pair, half) finishes rows half*8 .. half*8+7.
         const int pg = ft * 64 + pl;
         const bool want_img = p.img_out != nullptr;
         float keep0[8], keep1[8];  // results this thread owes the output image
 #pragma unroll
         for (int t8 = 0; t8 < 8; ++t8) {
+          const float own_lo = hi[t8], own_hi = hi[8 + t8];  // rows 0..7 and 8..15 of the chunk, this lane's feature
+          const float oth_lo = __shfl_xor_sync(0xffffffffu, own_lo, 16), oth_hi = __shfl_xor_sync(0xffffffffu, own_hi, 16);
+          float v0 = half ? oth_hi : own_lo, v1 = half ? own_hi : oth_lo;
           const int t = half * 8 + t8;
           const int m = row0 + c * kUmChunk + t;
-          float v0 = ex[pl * kUmExLd + t], v1 = ex[(pl + 64) * kUmExLd + t];
           keep0[t8] = 0.f;
           keep1[t8] = 0.f;
           if (m < p.M && pg < p.n_pairs) {
@@ -436,25 +451,28 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
             }
           }
         }
-        um_epi_sync();  // ex has been read
         if (want_img) {
-          // results back into ex as [feature of the tile][row], then 16-byte pieces of the image:
-          // 8 consecutive features of one row, high parts and low parts
+          // Results into this warp's own piece of shared memory as [feature][row], then out as 16-byte
+          // pieces of the image (8 consecutive features of one row, high parts and low parts).  A warp
+          // covers 32 consecutive features of the residual stream, or 16 consecutive columns of u.
           const bool resid = p.ep.mode == EPI_RESID;
-          const int f0 = resid ? ((pl >> 3) << 4) + (pl & 7) : pl;
+          float* exw = ex + quarter * (32 * kUmExLd);
+          const int li = lane & 15;
+          const int f0 = resid ? ((li >> 3) << 4) + (li & 7) : li;
+          __syncwarp();
 #pragma unroll
           for (int t8 = 0; t8 < 8; ++t8) {
-            ex[f0 * kUmExLd + half * 8 + t8] = keep0[t8];
-            if (resid) ex[(f0 + 8) * kUmExLd + half * 8 + t8] = keep1[t8];
+            exw[f0 * kUmExLd + half * 8 + t8] = keep0[t8];
+            if (resid) exw[(f0 + 8) * kUmExLd + half * 8 + t8] = keep1[t8];
           }
-          um_epi_sync();
-          const int t = et & 15, m = row0 + c * kUmChunk + t;
-          const int n_kg = resid ? 16 : 8, feat0 = ft * (resid ? 128 : 64);
+          __syncwarp();
+          const int t = lane & 15, m = row0 + c * kUmChunk + t;
+          const int n_kg = resid ? 4 : 2, feat0 = resid ? ft * 128 + quarter * 32 : ft * 64 + quarter * 16;
           if (m < p.M) {
-            for (int kgl = et >> 4; kgl < n_kg; kgl += 8) {
+            for (int kgl = lane >> 4; kgl < n_kg; kgl += 2) {
               float v[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) v[e] = ex[(kgl * 8 + e) * kUmExLd + t];
+              for (int e = 0; e < 8; ++e) v[e] = exw[(kgl * 8 + e) * kUmExLd + t];
               const int k0 = feat0 + kgl * 8;  // first feature of the piece = column of the next layer's input
               if (k0 >= p.img_KB * kUmBK) continue;
               if (p.gain_out != nullptr) {
@@ -472,15 +490,14 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
               *reinterpret_cast<uint4*>(dst + um_img_lo(RB)) = l4;
             }
           }
-          if (resid && p.ssq_out != nullptr && et < 16 && row0 + c * kUmChunk + et < p.M) {
-            float ssum = 0.f;  // this tile's 128 features of row et, in feature order
-            for (int fl = 0; fl < kUmFeat; ++fl) {
-              const float x = ex[fl * kUmExLd + et];
+          if (resid && p.ssq_out != nullptr && lane < 16 && m < p.M) {
+            float ssum = 0.f;  // this warp's 32 features of row `lane`, in feature order
+            for (int fl = 0; fl < 32; ++fl) {
+              const float x = exw[fl * kUmExLd + lane];
               ssum = fmaf(x, x, ssum);
             }
-            p.ssq_out[(size_t)ft * p.ssq_ld + row0 + c * kUmChunk + et] = ssum;
+            p.ssq_out[(size_t)(ft * 4 + quarter) * p.ssq_ld + m] = ssum;
           }
-          um_epi_sync();  // ex is rewritten by the next chunk
         }
       }
       // tensor memory of this accumulator has been read: hand it back to the MMA warp
@@ -510,8 +527,8 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
 
 // ---- operand images ---------------------------------------------------------------------------------
 // Weight image: element e of tile (ft, kb): k group j = e / 1024, row group i = (e % 1024) / 64, row
-// r8 = (e % 64) / 8, element e8 = e % 8; tile row R = 8 i + r8 is the first (R < 64) or second
-// feature of pair 64 ft + R % 64; column k = 64 kb + 8 j + e8.  Rows and columns beyond the matrix
+// r8 = (e % 64) / 8, element e8 = e % 8; tile row R = 8 i + r8 is the first (R % 32 < 16) or second
+// feature of pair 64 ft + 16 (R / 32) + R % 16; column k = 64 kb + 8 j + e8.  Rows and columns beyond the matrix
 // are zero.
 __global__ void pack_umma_kernel(__nv_bfloat16* __restrict__ dst, PackSrc ps, int n_pairs, int K, int n_ft, int KB) {
   const size_t total = (size_t)n_ft * KB * (kUmABytes / 2);
@@ -521,7 +538,7 @@ __global__ void pack_umma_kernel(__nv_bfloat16* __restrict__ dst, PackSrc ps, in
     const int ft = (int)(blk / KB), kb = (int)(blk % KB);
     const int j = w >> 10, i = (w >> 6) & 15, r8 = (w >> 3) & 7, e8 = w & 7;
     const int R = 8 * i + r8;
-    const int pr = ft * 64 + (R & 63), second = R >> 6;
+    const int pr = ft * 64 + 16 * (R >> 5) + (R & 15), second = (R >> 4) & 1;
     const int k = kb * kUmBK + 8 * j + e8;
     dst[e] = (pr < n_pairs && k < K) ? pack_src_row<__nv_bfloat16>(ps, pr, second, K)[k] : __float2bfloat16_rn(0.f);
   }

@@ -712,3 +712,20 @@ def test_kv_sharing_draft_batch_and_sampling():
         assert same >= 11
     finally:
         eng.close()
+
+
+def test_bf16_error_budget_against_unrounded_cache(tiny_bf16, l7b4, capsys):
+    """The bf16 configurations round K/V to bf16 on both sides (oracle and library).  Against an
+    oracle that keeps K/V in fp32 the library's logits must still sit inside the same tolerance;
+    both figures are printed (run with -s) so that the share of the K/V rounding is on record."""
+    import dataclasses
+    for name, (eng, m) in (("tiny-bf16", tiny_bf16), ("7b-4layers", l7b4)):
+        toks = si.make_prompts(m.vocab, 1, 100, seed=95)[0].tolist()
+        got = np.concatenate([eng.sdfp_forward_logits(toks[:64], 0), eng.sdfp_forward_logits(toks[64:], 64)])
+        same = orc.forward_nocache(m, toks).detach().numpy()
+        unrounded = orc.forward_nocache(dataclasses.replace(m, kv_bf16=False), toks).detach().numpy()
+        e_same, e_unr, e_kv = rel_l2(got, same), rel_l2(got, unrounded), rel_l2(same, unrounded)
+        with capsys.disabled():
+            print("\n[bf16 error budget] %s: library vs oracle (K/V rounded on both sides) %.3e; library vs oracle with fp32 K/V %.3e; "
+                  "the two oracles against each other %.3e" % (name, e_same, e_unr, e_kv))
+        assert e_same < 1e-2 and e_unr < 1e-2

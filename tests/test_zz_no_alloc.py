@@ -97,3 +97,18 @@ def test_static_call_allocates_nothing_and_leaves_the_context_intact():
     finally:
         eng.close()
         fresh.close()
+
+
+def test_static_scratch_on_the_dense_path():
+    """A context too wide for the whole-pass kernel decodes on the tcgen05 path, whose attention
+    kernel leaves a fixed 8 partials per (row, head): the static variant must size its array for
+    that and reproduce the ordinary entry point bit for bit, twice in a row."""
+    eng, m, _ = make_pair(si.TINY_BF16, (1, 2), max_seq=160, max_batch=4, k_max=4)
+    try:
+        toks = si.make_prompts(m.vocab, 1, 100, seed=27)[0].tolist()
+        for start, n in ((0, 72), (72, 9)):
+            ref = eng.sdfp_forward_logits(toks[start:start + n], start)
+            got = eng.sdfp_forward_logits_static(toks[start:start + n], start)
+            assert np.array_equal(got.view(np.uint32), ref.view(np.uint32))
+    finally:
+        eng.close()
