@@ -33,6 +33,7 @@
 #include "umma_linear.cuh"
 
 using namespace sdfp;
+static_assert(kAmaxRows == kPassMaxRows, "the partial-argmax array is indexed by the whole-pass kernel's rows");
 
 namespace {
 
@@ -105,6 +106,8 @@ struct sdfp_ctx {
   PassSync* psync = nullptr;
   ulonglong2* split_partials = nullptr;
   float* ssq_part = nullptr;
+  int2* amax_part = nullptr;  // greedy decision fused into the lm-head: (largest logit, index) per (group of the vocabulary, row)
+  int amax_groups = 0;
   int pass_slots[3] = {0, 0, 0};  // ring slots of the instantiation with 1 and with 2 column groups
   size_t pass_smem = 0;
   int pass_grid = 0;
@@ -472,7 +475,7 @@ cudaError_t launch_pass_t(sdfp_ctx* c, const PassParams& pp) {
 #define SDFP_PREFETCH_CHUNKS 8
 #endif
 
-cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool with_lm_head) {
+cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool with_lm_head, bool fused_argmax = false) {
   PassParams pp{};
   pp.prog = draft ? c->prog_d : c->prog_t;
   pp.n_stages = (draft ? c->n_prog_d : c->n_prog_t) - (with_lm_head ? 0 : 1);
@@ -488,6 +491,7 @@ cudaError_t run_pass(sdfp_ctx* c, bool draft, int rows, int rows_per_seq, bool w
   pp.part_ml = c->part_ml;
   pp.split_partials = c->split_partials;
   pp.ssq_part = c->ssq_part;
+  pp.amax_part = fused_argmax ? c->amax_part : nullptr;
   pp.sync = c->psync;
   const bool hd128 = c->cfg.head_dim == 128;
   if (rows <= 8) return hd128 ? launch_pass_t<1, 128>(c, pp) : launch_pass_t<1, 64>(c, pp);
@@ -520,7 +524,10 @@ int enqueue_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, int attn
   const KvCache& kv = (draft && !c->share_kv) ? c->cache_d : c->cache_t;
   const bool whole_pass = c->use_pass;  // a context takes ONE path for all its passes (see sdfp_create)
   if (whole_pass && rows > kPassMaxRows) return fail(c, SDFP_ESTATE, "a pass of %d rows reached the whole-pass kernel", rows);
-  if (whole_pass) CU_OK(c, run_pass(c, draft, rows, attn_rows_per_seq, decide != DECIDE_NONE));
+  // greedy decisions of the rounds are taken inside the pass kernel's lm-head (pd.amax_part set by enqueue_round)
+  const bool fused_argmax = whole_pass && decide == DECIDE_ARGMAX && pd.amax_part != nullptr;
+  if (whole_pass) CU_OK(c, run_pass(c, draft, rows, attn_rows_per_seq, decide != DECIDE_NONE, fused_argmax));
+  if (fused_argmax) return 0;
   for (int l = 0; l < g.n_layers && !whole_pass; ++l) {
     // Algorithm 1: pruned layers are removed from the draft, attention and FFN blocks separately
     const bool run_attn = !draft || c->keep_attn[l], run_ffn = !draft || c->keep_ffn[l];
@@ -641,6 +648,11 @@ int enqueue_dense_pass(sdfp_ctx* c, const PassDesc& pd, bool draft, int rows, in
 int enqueue_round(sdfp_ctx* c, int k, int batch, bool sampled, int n_chunks) {
   PassDesc pd{};
   pd.n_seq = batch;
+  const bool fused = c->use_pass && !sampled;  // the lm-head leaves argmax partials; consumers finish them
+  if (fused) {
+    pd.amax_part = c->amax_part;
+    pd.amax_groups = c->amax_groups;
+  }
   if (k > 0) {
     // The draft's own cache lags one token after a fully accepted round, so its first pass feeds
     // the last two committed tokens; a draft that shares the target's cache feeds the last one.
@@ -652,12 +664,14 @@ int enqueue_round(sdfp_ctx* c, int k, int batch, bool sampled, int n_chunks) {
     for (int s = 1; s < k; ++s) {
       pd.kind = PASS_DRAFT_NEXT;
       pd.step = s;
+      pd.prev_rows_per_seq = fused ? (s == 1 ? first_rows : 1) : 0;
       pd.rows_per_seq = 1;
       if (int r = enqueue_pass(c, pd, true, batch, 1, n_chunks, sampled ? DECIDE_SAMPLE_DRAFT : DECIDE_ARGMAX)) return r;
     }
   }
   pd.kind = PASS_VERIFY;
   pd.step = 0;
+  pd.prev_rows_per_seq = (fused && k > 0) ? (k == 1 ? (c->share_kv ? 1 : 2) : 1) : 0;
   pd.rows_per_seq = k + 1;
   if (int r = enqueue_pass(c, pd, false, (k + 1) * batch, k + 1, n_chunks, sampled ? DECIDE_LOGITS : DECIDE_ARGMAX))
     return r;
@@ -667,8 +681,9 @@ int enqueue_round(sdfp_ctx* c, int k, int batch, bool sampled, int n_chunks) {
                     c->cfg.vocab, (const int*)c->draft_tok, (const float*)c->qprob, (const double*)c->qsum, c->seq_tok,
                     c->cfg.max_seq, c->out_tok, c->stats, pass_err));
   else
-    CU_OK(c, launch(c, accept_greedy_kernel, dim3(1), dim3(32), 0, c->gs, (const int*)c->draft_tok,
-                    (const int*)c->tgt_tok, c->seq_tok, c->cfg.max_seq, c->out_tok, c->stats, pass_err));
+    CU_OK(c, launch(c, accept_greedy_kernel, dim3(1), dim3(kAcceptThreads), 0, c->gs, (const int*)c->draft_tok,
+                    (const int*)c->tgt_tok, c->seq_tok, c->cfg.max_seq, c->out_tok, c->stats, pass_err,
+                    (const int2*)(fused ? c->amax_part : nullptr), c->amax_groups));
   return 0;
 }
 
@@ -872,6 +887,7 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   // result independent of the pass it sits in, and speculative output equal to autoregressive
   // output bit for bit.
   const int widest = g.max_batch * std::max(g.k_max + 1, 2);
+  c->amax_groups = (g.vocab / 16 + kUnitTiles - 1) / kUnitTiles;
   c->use_pass = c->use_mma && !(g.flags & SDFP_FLAG_NO_PASS_KERNEL) && prop.cooperativeLaunch && g.d_model >= 64 &&
                 g.n_heads <= kPassMaxHeads && g.d_model / 128 + 1 <= kSsqMaxGroups && widest <= kPassMaxRows;
   int optin = 0;
@@ -962,7 +978,9 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   if (c->use_pass) {
     if ((r = dev_alloc(c, &c->psync, 1, true)) ||
         (r = dev_alloc(c, &c->split_partials, (size_t)c->pass_grid * kUnitTiles * 2 * 64, true)) ||
-        (r = dev_alloc(c, &c->ssq_part, (size_t)kSsqMaxGroups * kPassMaxRows, true)) || (r = build_programs(c)))
+        (r = dev_alloc(c, &c->ssq_part, (size_t)kSsqMaxGroups * kPassMaxRows, true)) ||
+        (r = dev_alloc(c, &c->amax_part, (size_t)((g.vocab / 16 + kUnitTiles - 1) / kUnitTiles) * kPassMaxRows, true)) ||
+        (r = build_programs(c)))
       return bail(r);
   }
   if (cudaMallocHost(reinterpret_cast<void**>(&c->pinned_flag), 64) != cudaSuccess) {
@@ -1479,12 +1497,12 @@ extern "C" int sdfp_time_pass(sdfp_ctx* c, int32_t draft, int32_t rows, int32_t 
   };
   for (int i = 0; i < 3 && err == cudaSuccess; ++i) {  // warm-up
     err = plan();
-    if (err == cudaSuccess) err = run_pass(c, draft != 0, rows, rows, true);
+    if (err == cudaSuccess) err = run_pass(c, draft != 0, rows, rows, true, true);
   }
   for (int i = 0; i < iters && err == cudaSuccess; ++i) {
     err = plan();  // fresh residual rows every time, outside the timed interval
     if (err == cudaSuccess) err = cudaEventRecord(ev[2 * i], c->stream);
-    if (err == cudaSuccess) err = run_pass(c, draft != 0, rows, rows, true);
+    if (err == cudaSuccess) err = run_pass(c, draft != 0, rows, rows, true, true);  // as in a greedy round: decision in the lm-head
     if (err == cudaSuccess) err = cudaEventRecord(ev[2 * i + 1], c->stream);
   }
   if (err == cudaSuccess) err = cudaStreamSynchronize(c->stream);

@@ -34,7 +34,41 @@ struct PassDesc {
   int kind, step, rows_per_seq, n_seq;
   int seq, start, count;  // PASS_TOKENS
   const int* src;         // PASS_TOKENS: device token ids
+  // Greedy decision fused into the lm-head (whole-pass kernel): the previous pass left, per row and
+  // per 128-feature group of the vocabulary, the largest logit and its index; the kernel that needs
+  // the token finishes the argmax.  prev_rows_per_seq = rows per sequence of that previous pass
+  // (0: tokens come from draft_tok / tgt_tok as written by argmax_kernel).
+  int prev_rows_per_seq;
+  const int2* amax_part;  // [group][kAmaxRows] (float bits, index)
+  int amax_groups;
 };
+
+constexpr int kAmaxRows = 16;  // rows per group in the partial-argmax array (the whole-pass kernel's row capacity)
+
+// Largest logit of row `row` over all groups, ties to the lowest index; one warp, every lane gets the result.
+__device__ __forceinline__ int amax_finish(const int2* part, int n_groups, int row) {
+  const int lane = threadIdx.x & 31;
+  float best = -INFINITY;
+  int bi = 0x7fffffff;
+  for (int g = lane; g < n_groups; g += 32) {
+    const int2 v = __ldcg(part + (size_t)g * kAmaxRows + row);
+    const float x = __int_as_float(v.x);
+    if (x > best || (x == best && v.y < bi)) {
+      best = x;
+      bi = v.y;
+    }
+  }
+#pragma unroll
+  for (int o = 16; o > 0; o >>= 1) {
+    const float ob = __shfl_xor_sync(0xffffffffu, best, o);
+    const int oi = __shfl_xor_sync(0xffffffffu, bi, o);
+    if (ob > best || (ob == best && oi < bi)) {
+      best = ob;
+      bi = oi;
+    }
+  }
+  return bi;
+}
 
 struct RowPlan {
   int* row_pos;  // [kMaxRows]
@@ -63,6 +97,19 @@ plan_embed_kernel(PassDesc pd, const GenState* gs, const int* seq_tok, int max_s
   pdl_wait();
   pdl_launch_dependents();
   const int m = blockIdx.x;
+  // a draft token the previous pass decided but nobody has written down yet (fused argmax)
+  int pending = -1;
+  if (pd.prev_rows_per_seq > 0 && threadIdx.x < 32) {
+    const int R = pd.rows_per_seq;
+    const int b = m / R, i = m - b * R;
+    const bool mine = (pd.kind == PASS_DRAFT_NEXT) || (pd.kind == PASS_VERIFY && R > 1 && i == R - 1);
+    if (mine && !ld_act(&gs->done[b])) {
+      const int pr = pd.prev_rows_per_seq;
+      pending = amax_finish(pd.amax_part, pd.amax_groups, b * pr + pr - 1);
+      const int slot = (pd.kind == PASS_DRAFT_NEXT) ? pd.step - 1 : R - 2;
+      if (threadIdx.x == 0) const_cast<int*>(draft_tok)[b * kMaxK + slot] = pending;
+    }
+  }
   if (threadIdx.x == 0) {
     int tok = 0, pos = -1, seq = 0;
     if (pd.kind == PASS_TOKENS) {
@@ -82,10 +129,11 @@ plan_embed_kernel(PassDesc pd, const GenState* gs, const int* seq_tok, int max_s
           if (pos >= 0) tok = ld_act(seq_tok + (size_t)b * max_seq + pos);
         } else if (pd.kind == PASS_DRAFT_NEXT) {
           pos = n - 1 + pd.step;
-          tok = ld_act(draft_tok + b * kMaxK + pd.step - 1);
+          tok = pending >= 0 ? pending : ld_act(draft_tok + b * kMaxK + pd.step - 1);
         } else {
           pos = n - 1 + i;
-          tok = (i == 0) ? ld_act(seq_tok + (size_t)b * max_seq + n - 1) : ld_act(draft_tok + b * kMaxK + i - 1);
+          tok = (i == 0) ? ld_act(seq_tok + (size_t)b * max_seq + n - 1)
+                         : (pending >= 0 ? pending : ld_act(draft_tok + b * kMaxK + i - 1));
         }
       }
     }
@@ -223,23 +271,34 @@ __device__ __forceinline__ void commit_tokens(volatile GenState* gs, int b, int 
 
 // Greedy accept (Eq. 2 degenerates to "draft token == target argmax"); k = 0 is a
 // plain autoregressive step.
-__global__ void __launch_bounds__(32)
+constexpr int kAcceptThreads = 256;
+__global__ void __launch_bounds__(kAcceptThreads)
 accept_greedy_kernel(GenState* gs_, const int* draft_tok, const int* tgt_tok, int* seq_tok, int max_seq,
-                     int* out_tok, RoundStat* stats, const int* pass_error) {
+                     int* out_tok, RoundStat* stats, const int* pass_error, const int2* amax_part, int amax_groups) {
   volatile GenState* gs = gs_;
+  __shared__ int s_tgt[kMaxBatch * (kMaxK + 1)];
   pdl_wait();
   pdl_launch_dependents();
-  const int b = threadIdx.x;
   const int B = gs->batch, k = gs->k;
+  // the target's argmax of every verify row: finished here from the lm-head's per-group partials
+  // (whole-pass kernel), else read where argmax_kernel left it
+  for (int r = threadIdx.x >> 5; r < B * (k + 1); r += kAcceptThreads / 32) {
+    const int b2 = r / (k + 1), i2 = r - b2 * (k + 1);
+    const int v = amax_part ? amax_finish(amax_part, amax_groups, r) : ld_act(tgt_tok + b2 * (kMaxK + 1) + i2);
+    if ((threadIdx.x & 31) == 0) s_tgt[b2 * (kMaxK + 1) + i2] = v;
+  }
+  __syncthreads();
+  if (threadIdx.x >= 32) return;
+  const int b = threadIdx.x;
   if (b < B) {
     if (gs->done[b]) {
       if (gs->round < gs->max_rounds) stats[(size_t)gs->round * B + b] = RoundStat{0, 0, 0};
     } else {
       const int* d = draft_tok + b * kMaxK;
-      const int* t = tgt_tok + b * (kMaxK + 1);
+      const int* t = s_tgt + b * (kMaxK + 1);
       int j = 0;
-      while (j < k && ld_act(d + j) == ld_act(t + j)) ++j;
-      commit_tokens(gs, b, k, j, ld_act(t + j), d, seq_tok, max_seq, out_tok, stats);
+      while (j < k && ld_act(d + j) == t[j]) ++j;
+      commit_tokens(gs, b, k, j, t[j], d, seq_tok, max_seq, out_tok, stats);
     }
   }
   __syncwarp();

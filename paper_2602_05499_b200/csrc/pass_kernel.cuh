@@ -118,6 +118,10 @@ struct PassParams {
   float* part_ml;         // [rows][head][kAttnSplits][2] running max and sum
   ulonglong2* split_partials;  // [grid][kUnitTiles * CG * 64] packets of two (value, stage serial) words
   float* ssq_part;        // [kSsqMaxGroups][kPassMaxRows]
+  // Greedy decision fused into the lm-head: non-null = the EPI_LOGITS stage writes no logits but,
+  // per (128-feature group, row), the largest logit and its index (ties: lowest index); whoever
+  // needs the token takes the maximum over the groups (amax_finish in misc_kernels.cuh).
+  int2* amax_part;        // [groups of the vocabulary][kPassMaxRows]
   PassSync* sync;
 };
 
@@ -383,6 +387,8 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
   float4* red = reinterpret_cast<float4*>(work);
   float* sq_buf = reinterpret_cast<float*>(work + work_sq_off<CG>());
   float* sc = reinterpret_cast<float*>(work + work_sc_off<CG>());
+  const bool fused_argmax = st.ep.mode == EPI_LOGITS && pp.amax_part != nullptr;
+  int* idx_buf = reinterpret_cast<int*>(sc);  // the lm-head reads plain activations: the fold area is free
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int g = lane >> 2, q = lane & 3;
   const int cls = warp & (kClasses - 1), th = warp / kClasses;
@@ -694,11 +700,19 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
             hp[0] = n0;
             hp[8] = n1;
             sq = fmaf(n0, n0, n1 * n1);
+          } else if (fused_argmax) {
+            const float a = v0 * inv, b2 = v1 * inv;  // logits of features 16 rt + ln/4 and + 8
+            const int f0 = 16 * rt + (ln >> 2);
+            sq = b2 > a ? b2 : a;
+            idx_buf[it] = b2 > a ? f0 + 8 : f0;
           } else {
             apply_epilogue<__nv_bfloat16>(st.ep, 8 * rt + (ln >> 2), m, v0 * inv, v1 * inv);
           }
+        } else if (fused_argmax) {
+          sq = -INFINITY;
+          idx_buf[it] = 0x7fffffff;
         }
-        if (st.write_ssq) sq_buf[it] = sq;
+        if (st.write_ssq || fused_argmax) sq_buf[it] = sq;
       }
     }
     if (starts_group && st.write_ssq) {
@@ -710,6 +724,26 @@ __device__ void linear_stage(const PassParams& pp, PassShared* sh, const unsigne
         for (int tile = 0; tile < kUnitTiles; ++tile)
           for (int g8 = 0; g8 < 8; ++g8) s += sq_buf[(((tile * CG + cg) * 32) + g8 * 4 + qq) * 2 + ch];
         pp.ssq_part[grp * kPassMaxRows + tid] = s;
+      }
+    }
+    if (starts_group && fused_argmax) {
+      // the group's best logit per row, candidates in tile-then-row order, ties to the lowest index
+      consumer_sync();
+      if (tid < M) {
+        const int cg = tid >> 3, qq = (tid & 7) >> 1, ch = tid & 1;
+        float best = -INFINITY;
+        int bi = 0x7fffffff;
+        for (int tile = 0; tile < kUnitTiles; ++tile)
+          for (int g8 = 0; g8 < 8; ++g8) {
+            const int e = (((tile * CG + cg) * 32) + g8 * 4 + qq) * 2 + ch;
+            const float x = sq_buf[e];
+            const int xi = idx_buf[e];
+            if (x > best || (x == best && xi < bi)) {
+              best = x;
+              bi = xi;
+            }
+          }
+        pp.amax_part[grp * kPassMaxRows + tid] = make_int2(__float_as_int(best), bi);
       }
     }
     consumer_sync();  // red and parts may be rewritten
