@@ -238,6 +238,27 @@ int sdfp_forward_logits(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int
 int sdfp_forward_logits_static(sdfp_ctx *ctx, int32_t draft, const int32_t *tokens, int32_t rows,
                                int32_t start, float *host_logits);
 
+/*
+ * Stage A of Algorithm 1 ("FIT-based pruning"): the layer scores from which the prune set P is
+ * chosen.  No context is needed; the weights are read where the caller has them (same structure
+ * and storage type as for sdfp_create, row-major [out, in]) and nothing is kept.
+ *   tokens     host int32 [n_seq, seq_len]: the calibration set D, one sequence = one sample z_i;
+ *              f(z_i, theta) = mean cross-entropy of token t+1 under the logits at position t
+ *   out_trace  host double [n_layers]: T_l = (1/N) sum_i ||grad_{theta_l} f(z_i, theta)||^2, the
+ *              empirical-Fisher trace of layer l (Eq. 11; Eq. 8-9), over the layer's seven
+ *              matrices and two norm gains
+ *   out_fit    host double [n_layers] or NULL: sum over the layer's tensors of T_t * mean(theta_t^2),
+ *              the layer-wise FIT form (Eq. 7) with the perturbation of removing the layer,
+ *              delta theta = -theta
+ * Algorithm 1 then sorts ascending and prunes the floor(r L) lowest layers; feed the result to
+ * sdfp_set_draft_layers.  One forward and one backward pass per sequence in fp32 (squared norms
+ * accumulated in fp64); device memory for the activations of one sequence is allocated and freed
+ * inside the call, which is synchronous.  Errors as for sdfp_create (message via
+ * sdfp_last_error(NULL)).
+ */
+int sdfp_fit_scores(const sdfp_config *cfg, const sdfp_weights *w, void *cuda_stream, const int32_t *tokens,
+                    int32_t n_seq, int32_t seq_len, double *out_trace, double *out_fit);
+
 /* Timing of the last successful sdfp_generate. */
 int sdfp_get_timing(const sdfp_ctx *ctx, sdfp_timing *out);
 

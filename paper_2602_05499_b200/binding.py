@@ -17,7 +17,7 @@ FLAG_NO_GRAPH, FLAG_NO_PDL, FLAG_FMA_GEMM, FLAG_NO_PASS_KERNEL, FLAG_NO_DENSE = 
 
 EXPORTS = ["sdfp_create", "sdfp_set_draft_layers", "sdfp_set_draft_sublayers", "sdfp_set_draft_kv_sharing", "sdfp_generate", "sdfp_forward_logits",
            "sdfp_forward_logits_static", "sdfp_get_timing", "sdfp_time_linear", "sdfp_time_pass",
-           "sdfp_debug_expire_next_wait", "sdfp_last_error", "sdfp_destroy"]
+           "sdfp_debug_expire_next_wait", "sdfp_fit_scores", "sdfp_last_error", "sdfp_destroy"]
 
 
 class SdfpConfig(C.Structure):
@@ -94,6 +94,9 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     lib.sdfp_time_pass.restype = C.c_int
     lib.sdfp_debug_expire_next_wait.argtypes = [vp, C.c_uint64]
     lib.sdfp_debug_expire_next_wait.restype = C.c_int
+    lib.sdfp_fit_scores.argtypes = [C.POINTER(SdfpConfig), C.POINTER(SdfpWeights), vp, C.POINTER(C.c_int32), C.c_int32, C.c_int32,
+                                    C.POINTER(C.c_double), C.POINTER(C.c_double)]
+    lib.sdfp_fit_scores.restype = C.c_int
     lib.sdfp_last_error.argtypes = [vp]
     lib.sdfp_last_error.restype = C.c_char_p
     lib.sdfp_destroy.argtypes = [vp]
@@ -101,6 +104,52 @@ def load_library(path: Optional[str] = None) -> C.CDLL:
     if path is None:
         _lib = lib
     return lib
+
+
+def _marshal(shape, weights: Dict, max_seq: int, max_batch: int, k_max: int, eos_id: int, flags: int):
+    """(SdfpConfig, SdfpWeights, objects that must stay alive) for a dict of CUDA tensors."""
+    import torch
+    want = torch.float32 if shape.dtype == "f32" else torch.bfloat16
+    L = shape.n_layers
+
+    def ptr(t):
+        if not t.is_cuda or t.dtype != want or not t.is_contiguous():
+            raise ValueError("weights must be contiguous CUDA tensors of the model's storage type")
+        return t.data_ptr()
+
+    arrs = {}
+    for name in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "attn_norm", "ffn_norm"):
+        arrs[name] = (C.c_void_p * L)(*[ptr(weights["layers"][l][name]) for l in range(L)])
+    w = SdfpWeights(ptr(weights["tok_embed"]), ptr(weights["final_norm"]), ptr(weights["lm_head"]),
+                    *[C.cast(arrs[n], C.POINTER(C.c_void_p)) for n in
+                      ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "attn_norm", "ffn_norm")])
+    cfg = SdfpConfig(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn,
+                     shape.vocab, shape.rms_eps, shape.rope_theta, max_seq, max_batch, k_max,
+                     SDFP_F32 if shape.dtype == "f32" else SDFP_BF16, eos_id, flags)
+    return cfg, w, arrs
+
+
+def sdfp_fit_scores(shape, weights: Dict, calib) -> "tuple":
+    """Stage A of Algorithm 1 on the GPU: (T_l, FIT_l) per layer over the calibration sequences
+    `calib` (int array [n_seq, seq_len]).  Argument marshalling only."""
+    import torch
+    if not torch.cuda.is_available():
+        raise RuntimeError("no CUDA device: the SDFP library has no CPU path")
+    lib = load_library()
+    cfg, w, keep = _marshal(shape, weights, 8, 1, 0, -1, 0)
+    t = np.ascontiguousarray(np.asarray(calib, dtype=np.int32))
+    if t.ndim != 2:
+        raise ValueError("calib must be [n_seq, seq_len]")
+    trace = np.zeros(shape.n_layers, dtype=np.float64)
+    fit = np.zeros(shape.n_layers, dtype=np.float64)
+    torch.cuda.current_stream().synchronize()
+    rc = lib.sdfp_fit_scores(C.byref(cfg), C.byref(w), C.c_void_p(torch.cuda.current_stream().cuda_stream),
+                             t.ctypes.data_as(C.POINTER(C.c_int32)), t.shape[0], t.shape[1],
+                             trace.ctypes.data_as(C.POINTER(C.c_double)), fit.ctypes.data_as(C.POINTER(C.c_double)))
+    if rc != 0:
+        raise SdfpError(rc, lib.sdfp_last_error(None).decode())
+    del keep
+    return trace.tolist(), fit.tolist()
 
 
 class GenOutput:
@@ -134,23 +183,7 @@ class Sdfp:
         self.lib = load_library()
         self.shape = shape
         self._stream = stream if stream is not None else torch.cuda.Stream()
-        want = torch.float32 if shape.dtype == "f32" else torch.bfloat16
-        L = shape.n_layers
-
-        def ptr(t):
-            if not t.is_cuda or t.dtype != want or not t.is_contiguous():
-                raise ValueError("weights must be contiguous CUDA tensors of the model's storage type")
-            return t.data_ptr()
-
-        arrs = {}
-        for name in ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "attn_norm", "ffn_norm"):
-            arrs[name] = (C.c_void_p * L)(*[ptr(weights["layers"][l][name]) for l in range(L)])
-        w = SdfpWeights(ptr(weights["tok_embed"]), ptr(weights["final_norm"]), ptr(weights["lm_head"]),
-                        *[C.cast(arrs[n], C.POINTER(C.c_void_p)) for n in
-                          ("wq", "wk", "wv", "wo", "w_gate", "w_up", "w_down", "attn_norm", "ffn_norm")])
-        cfg = SdfpConfig(shape.n_layers, shape.d_model, shape.n_heads, shape.head_dim, shape.d_ffn,
-                         shape.vocab, shape.rms_eps, shape.rope_theta, max_seq, max_batch, k_max,
-                         SDFP_F32 if shape.dtype == "f32" else SDFP_BF16, eos_id, flags)
+        cfg, w, self._keep = _marshal(shape, weights, max_seq, max_batch, k_max, eos_id, flags)
         self.cfg = cfg
         handle = C.c_void_p()
         # the caller's tensors were produced on torch's current stream

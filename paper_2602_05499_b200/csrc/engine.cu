@@ -24,6 +24,7 @@
 #include "attention.cuh"
 #include "common.cuh"
 #include "dense_attention.cuh"
+#include "fit.cuh"
 #include "linear_fma.cuh"
 #include "linear_mma.cuh"
 #include "misc_kernels.cuh"
@@ -1461,6 +1462,38 @@ extern "C" int sdfp_debug_expire_next_wait(sdfp_ctx* c, uint64_t wait_limit_ns) 
   const unsigned long long words[2] = {1ull, (unsigned long long)wait_limit_ns};  // bar_extra, wait_limit_ns
   CU_OK(c, cudaMemcpyAsync(&c->psync->bar_extra, words, sizeof words, cudaMemcpyHostToDevice, c->stream));
   CU_OK(c, cudaStreamSynchronize(c->stream));  // words is a local
+  return 0;
+}
+
+extern "C" int sdfp_fit_scores(const sdfp_config* cfg, const sdfp_weights* w, void* cuda_stream, const int32_t* tokens,
+                               int32_t n_seq, int32_t seq_len, double* out_trace, double* out_fit) {
+  if (!cfg || !w || !tokens || !out_trace) return fail(nullptr, SDFP_EINVAL, "sdfp_fit_scores: NULL argument");
+  const sdfp_config& g = *cfg;
+  if (g.n_layers < 1 || g.n_layers > 1024 || g.d_model < 2 || g.n_heads < 1 || g.d_ffn < 1 || g.vocab < 2 || g.head_dim < 2 ||
+      (g.head_dim & 1) || g.d_model != g.n_heads * g.head_dim)
+    return fail(nullptr, SDFP_EINVAL, "sdfp_fit_scores: bad model dimensions");
+  if (g.dtype != SDFP_F32 && g.dtype != SDFP_BF16) return fail(nullptr, SDFP_EINVAL, "unknown dtype");
+  if (!(g.rms_eps > 0.f) || !(g.rope_theta > 0.f)) return fail(nullptr, SDFP_EINVAL, "bad rms_eps or rope_theta");
+  if (n_seq < 1 || seq_len < 2 || seq_len > 4097) return fail(nullptr, SDFP_EINVAL, "sdfp_fit_scores: need n_seq >= 1 and 2 <= seq_len <= 4097");
+  if (!w->tok_embed || !w->final_norm || !w->lm_head || !w->wq || !w->wk || !w->wv || !w->wo || !w->w_gate || !w->w_up || !w->w_down ||
+      !w->attn_norm || !w->ffn_norm)
+    return fail(nullptr, SDFP_EINVAL, "sdfp_fit_scores: NULL weight pointer");
+  for (int l = 0; l < g.n_layers; ++l)
+    if (!w->wq[l] || !w->wk[l] || !w->wv[l] || !w->wo[l] || !w->w_gate[l] || !w->w_up[l] || !w->w_down[l] || !w->attn_norm[l] ||
+        !w->ffn_norm[l])
+      return fail(nullptr, SDFP_EINVAL, "layer %d has a NULL weight pointer", l);
+  for (int64_t i = 0; i < (int64_t)n_seq * seq_len; ++i)
+    if (tokens[i] < 0 || tokens[i] >= g.vocab) return fail(nullptr, SDFP_EINVAL, "calibration token %d out of range", tokens[i]);
+  int ndev = 0;
+  if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev == 0) {
+    cudaGetLastError();
+    return fail(nullptr, SDFP_ECUDA, "no CUDA device: this library has no CPU path");
+  }
+  cudaStream_t st = reinterpret_cast<cudaStream_t>(cuda_stream);
+  const cudaError_t e = g.dtype == SDFP_BF16 ? fit::run<__nv_bfloat16>(g, w, st, tokens, n_seq, seq_len, out_trace, out_fit)
+                                              : fit::run<float>(g, w, st, tokens, n_seq, seq_len, out_trace, out_fit);
+  if (e != cudaSuccess)
+    return fail(nullptr, e == cudaErrorMemoryAllocation ? SDFP_ENOMEM : SDFP_ECUDA, "sdfp_fit_scores: %s", cudaGetErrorString(e));
   return 0;
 }
 
