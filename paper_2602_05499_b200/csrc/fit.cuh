@@ -14,7 +14,7 @@
 //
 // Everything is fp32 on CUDA cores with fp64 accumulation of the squared norms; weights are read in
 // their storage type (fp32 or bf16) from the caller's row-major [out, in] matrices.  This is the
-// offline, one-shot stage of the method: the kernels are plain (tiled GEMMs through shared memory,
+// offline, one-shot stage of the method: the kernels are plain (register-tiled GEMMs through shared memory,
 // one block per (row, head) in attention) and every reduction runs in a fixed order, so the scores
 // are reproducible bit for bit.
 #pragma once
@@ -29,48 +29,86 @@
 namespace sdfp {
 namespace fit {
 
-constexpr int kTile = 32;
 
 __device__ __forceinline__ float wload(const float* p) { return *p; }
 __device__ __forceinline__ float wload(const __nv_bfloat16* p) { return __bfloat162float(*p); }
 
+// Tiled fp32 GEMMs: a 64 x 64 output tile per block of 256 threads, 4 x 4 outputs per thread, the
+// contraction in steps of 16 through shared memory.  Rows (tokens) are few (a calibration sequence),
+// so every weight is read once per GEMM.
+constexpr int kGT = 64, kGK = 16;
+
 // C[T, N] = A[T, K] * W[N, K]^T
 template <typename WT>
-__global__ void __launch_bounds__(kTile * kTile) gemm_nt_kernel(const float* __restrict__ A, const WT* __restrict__ W,
-                                                                 float* __restrict__ C, int T, int N, int K) {
-  __shared__ float sA[kTile][kTile + 1], sW[kTile][kTile + 1];
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const int t = blockIdx.y * kTile + ty, n = blockIdx.x * kTile + tx;
-  float acc = 0.f;
-  for (int k0 = 0; k0 < K; k0 += kTile) {
-    sA[ty][tx] = (t < T && k0 + tx < K) ? A[(size_t)t * K + k0 + tx] : 0.f;
-    const int wn = blockIdx.x * kTile + ty;
-    sW[ty][tx] = (wn < N && k0 + tx < K) ? wload(W + (size_t)wn * K + k0 + tx) : 0.f;
+__global__ void __launch_bounds__(256) gemm_nt_kernel(const float* __restrict__ A, const WT* __restrict__ W, float* __restrict__ C,
+                                                       int T, int N, int K) {
+  __shared__ __align__(16) float sA[kGK][kGT + 4], sW[kGK][kGT + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int t0 = blockIdx.y * kGT, n0 = blockIdx.x * kGT;
+  float acc[4][4] = {};
+  for (int k0 = 0; k0 < K; k0 += kGK) {
+    for (int e = tid; e < kGT * kGK; e += 256) {  // element (row r, column kk): consecutive threads along k
+      const int r = e >> 4, kk = e & 15;
+      sA[kk][r] = (t0 + r < T && k0 + kk < K) ? A[(size_t)(t0 + r) * K + k0 + kk] : 0.f;
+      sW[kk][r] = (n0 + r < N && k0 + kk < K) ? wload(W + (size_t)(n0 + r) * K + k0 + kk) : 0.f;
+    }
     __syncthreads();
 #pragma unroll
-    for (int k = 0; k < kTile; ++k) acc = fmaf(sA[ty][k], sW[tx][k], acc);
+    for (int kk = 0; kk < kGK; ++kk) {
+      const float4 a = *reinterpret_cast<const float4*>(&sA[kk][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&sW[kk][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j2 = 0; j2 < 4; ++j2) acc[i][j2] = fmaf(av[i], bv[j2], acc[i][j2]);
+    }
     __syncthreads();
   }
-  if (t < T && n < N) C[(size_t)t * N + n] = acc;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j2 = 0; j2 < 4; ++j2) {
+      const int t = t0 + ty * 4 + i, n = n0 + tx * 4 + j2;
+      if (t < T && n < N) C[(size_t)t * N + n] = acc[i][j2];
+    }
 }
 
 // C[T, K] (+)= A[T, N] * W[N, K]     (the gradient of a linear layer's input)
 template <typename WT>
-__global__ void __launch_bounds__(kTile * kTile) gemm_nn_kernel(const float* __restrict__ A, const WT* __restrict__ W,
-                                                                 float* __restrict__ C, int T, int N, int K, int accumulate) {
-  __shared__ float sA[kTile][kTile + 1], sW[kTile][kTile + 1];
-  const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
-  const int t = blockIdx.y * kTile + ty, k = blockIdx.x * kTile + tx;
-  float acc = 0.f;
-  for (int n0 = 0; n0 < N; n0 += kTile) {
-    sA[ty][tx] = (t < T && n0 + tx < N) ? A[(size_t)t * N + n0 + tx] : 0.f;
-    sW[ty][tx] = (n0 + ty < N && k < K) ? wload(W + (size_t)(n0 + ty) * K + k) : 0.f;
+__global__ void __launch_bounds__(256) gemm_nn_kernel(const float* __restrict__ A, const WT* __restrict__ W, float* __restrict__ C,
+                                                       int T, int N, int K, int accumulate) {
+  __shared__ __align__(16) float sA[kGK][kGT + 4], sW[kGK][kGT + 4];
+  const int tid = threadIdx.x, tx = tid & 15, ty = tid >> 4;
+  const int t0 = blockIdx.y * kGT, c0 = blockIdx.x * kGT;
+  float acc[4][4] = {};
+  for (int n0 = 0; n0 < N; n0 += kGK) {
+    for (int e = tid; e < kGT * kGK; e += 256) {
+      const int r = e >> 4, nn = e & 15;  // A: (row r, contraction index nn), consecutive threads along n
+      sA[nn][r] = (t0 + r < T && n0 + nn < N) ? A[(size_t)(t0 + r) * N + n0 + nn] : 0.f;
+      const int wn = e >> 6, wc = e & 63;  // W: (contraction index wn, column wc), consecutive threads along the row
+      sW[wn][wc] = (n0 + wn < N && c0 + wc < K) ? wload(W + (size_t)(n0 + wn) * K + c0 + wc) : 0.f;
+    }
     __syncthreads();
 #pragma unroll
-    for (int n = 0; n < kTile; ++n) acc = fmaf(sA[ty][n], sW[n][tx], acc);
+    for (int nn = 0; nn < kGK; ++nn) {
+      const float4 a = *reinterpret_cast<const float4*>(&sA[nn][ty * 4]);
+      const float4 b = *reinterpret_cast<const float4*>(&sW[nn][tx * 4]);
+      const float av[4] = {a.x, a.y, a.z, a.w}, bv[4] = {b.x, b.y, b.z, b.w};
+#pragma unroll
+      for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j2 = 0; j2 < 4; ++j2) acc[i][j2] = fmaf(av[i], bv[j2], acc[i][j2]);
+    }
     __syncthreads();
   }
-  if (t < T && k < K) C[(size_t)t * K + k] = (accumulate ? C[(size_t)t * K + k] : 0.f) + acc;
+#pragma unroll
+  for (int i = 0; i < 4; ++i)
+#pragma unroll
+    for (int j2 = 0; j2 < 4; ++j2) {
+      const int t = t0 + ty * 4 + i, c = c0 + tx * 4 + j2;
+      if (t < T && c < K) C[(size_t)t * K + c] = (accumulate ? C[(size_t)t * K + c] : 0.f) + acc[i][j2];
+    }
 }
 
 // fixed-order block sum (blockDim.x a multiple of 32, at most 1024); every thread gets the result
@@ -324,17 +362,25 @@ __global__ void __launch_bounds__(256) gram_dot_kernel(const double* __restrict_
   const double tot = block_sum_d(s, s_red);
   if (threadIdx.x == 0) *out += tot;
 }
-// out = mean of w^2 over n elements; one block
+// mean of w^2 over n elements in two fixed-order steps: per-block partial sums, then one block adds them
+constexpr int kMsBlocks = 592;
 template <typename WT>
-__global__ void __launch_bounds__(256) mean_sq_kernel(const WT* __restrict__ w, size_t n, double* out) {
+__global__ void __launch_bounds__(256) sum_sq_partial_kernel(const WT* __restrict__ w, size_t n, double* __restrict__ partial) {
   __shared__ double s_red[8];
   double s = 0.0;
-  for (size_t i = threadIdx.x; i < n; i += blockDim.x) {
+  for (size_t i = (size_t)blockIdx.x * blockDim.x + threadIdx.x; i < n; i += (size_t)gridDim.x * blockDim.x) {
     const double v = wload(w + i);
     s += v * v;
   }
   const double tot = block_sum_d(s, s_red);
-  if (threadIdx.x == 0) *out = tot / (double)n;
+  if (threadIdx.x == 0) partial[blockIdx.x] = tot;
+}
+__global__ void __launch_bounds__(256) mean_finish_kernel(const double* __restrict__ partial, int n_part, double n, double* out) {
+  __shared__ double s_red[8];
+  double s = 0.0;
+  for (int i = threadIdx.x; i < n_part; i += blockDim.x) s += partial[i];
+  const double tot = block_sum_d(s, s_red);
+  if (threadIdx.x == 0) *out = tot / n;
 }
 
 // ---- host side --------------------------------------------------------------------------------------
@@ -384,6 +430,7 @@ cudaError_t run(const sdfp_config& g, const sdfp_weights* w, cudaStream_t st, co
   float *du = A.get<float>(Tf), *dgt = A.get<float>(Tf), *dup = A.get<float>(Tf);
   double *G1 = A.get<double>((size_t)T * T), *G2 = A.get<double>((size_t)T * T);
   double *sq = A.get<double>((size_t)L * kTensors), *msq = A.get<double>((size_t)L * kTensors);
+  double* ms_part = A.get<double>(kMsBlocks);
   int* tok = A.get<int>(seq_len);
   float *cs = A.get<float>((size_t)T * (hd / 2)), *sn = A.get<float>((size_t)T * (hd / 2));
   if (A.err != cudaSuccess) return A.err;
@@ -403,12 +450,11 @@ cudaError_t run(const sdfp_config& g, const sdfp_weights* w, cudaStream_t st, co
     FIT_OK(cudaStreamSynchronize(st));
   }
   auto W = [&](const void* const* arr, int l) { return reinterpret_cast<const WT*>(arr[l]); };
-  const dim3 gb(kTile * kTile);
   auto nt = [&](const float* Ain, const WT* Wm, float* C, int N, int K) {  // C[T,N] = A[T,K] W[N,K]^T
-    gemm_nt_kernel<WT><<<dim3((N + kTile - 1) / kTile, (T + kTile - 1) / kTile), gb, 0, st>>>(Ain, Wm, C, T, N, K);
+    gemm_nt_kernel<WT><<<dim3((N + kGT - 1) / kGT, (T + kGT - 1) / kGT), 256, 0, st>>>(Ain, Wm, C, T, N, K);
   };
   auto nn = [&](const float* Ain, const WT* Wm, float* C, int N, int K, int acc) {  // C[T,K] (+)= A[T,N] W[N,K]
-    gemm_nn_kernel<WT><<<dim3((K + kTile - 1) / kTile, (T + kTile - 1) / kTile), gb, 0, st>>>(Ain, Wm, C, T, N, K, acc);
+    gemm_nn_kernel<WT><<<dim3((K + kGT - 1) / kGT, (T + kGT - 1) / kGT), 256, 0, st>>>(Ain, Wm, C, T, N, K, acc);
   };
   auto gram = [&](const float* Ain, int n, double* G) { gram_kernel<<<dim3(T, T), 128, 0, st>>>(Ain, n, T, G); };
   auto gdot = [&](int l, int tensor) { gram_dot_kernel<<<1, 256, 0, st>>>(G1, G2, T * T, sq + (size_t)l * kTensors + tensor); };
@@ -485,8 +531,10 @@ cudaError_t run(const sdfp_config& g, const sdfp_weights* w, cudaStream_t st, co
   for (int l = 0; l < L; ++l) {
     const void* ptr[kTensors] = {w->wq[l], w->wk[l], w->wv[l], w->wo[l], w->w_gate[l], w->w_up[l], w->w_down[l], w->attn_norm[l], w->ffn_norm[l]};
     const size_t n[kTensors] = {(size_t)d * d, (size_t)d * d, (size_t)d * d, (size_t)d * d, (size_t)f * d, (size_t)f * d, (size_t)d * f, (size_t)d, (size_t)d};
-    for (int t = 0; t < kTensors; ++t)
-      mean_sq_kernel<WT><<<1, 256, 0, st>>>(reinterpret_cast<const WT*>(ptr[t]), n[t], msq + (size_t)l * kTensors + t);
+    for (int t = 0; t < kTensors; ++t) {
+      sum_sq_partial_kernel<WT><<<kMsBlocks, 256, 0, st>>>(reinterpret_cast<const WT*>(ptr[t]), n[t], ms_part);
+      mean_finish_kernel<<<1, 256, 0, st>>>(ms_part, kMsBlocks, (double)n[t], msq + (size_t)l * kTensors + t);
+    }
   }
   FIT_OK(cudaGetLastError());
   std::vector<double> hsq((size_t)L * kTensors), hms((size_t)L * kTensors);
