@@ -30,9 +30,9 @@
 // result does not depend on timing.  A row's result depends on its own column only.
 //
 // Roles: warp 0 = producer (bulk copies into a ring of stages, mbarrier transaction counts),
-// warp 1 = MMA issue (one thread) and owner of the tensor-memory allocation, warps 2..5 = epilogue
-// (tcgen05.ld, pair exchange through shared memory, the same fused epilogues as the other linear
-// kernels).  Two accumulators alternate, so the epilogue of one piece overlaps the MMAs of the next.
+// warp 1 = MMA issue (one thread) and owner of the tensor-memory allocation, warps 2..9 = epilogue
+// (two per quarter of tensor memory, one for the even and one for the odd 16-row chunks: tcgen05.ld,
+// pair partner by a shuffle, the same fused epilogues as the other linear kernels).  Two accumulators alternate, so the epilogue of one piece overlaps the MMAs of the next.
 // Every wait is bounded: a wait that runs out records an error word and the CTA winds down.
 #pragma once
 
@@ -46,8 +46,9 @@ constexpr int kUmBK = 64;                          // k elements per pipeline st
 constexpr int kUmFeat = 128;                       // output features per tile = tensor-memory lanes
 constexpr int kUmABytes = kUmFeat * kUmBK * 2;     // weight bytes per stage
 constexpr int kUmMaxRB = 128;                      // rows per row block (N = 2 * RB <= 256)
-constexpr int kUmThreads = 192;
-constexpr int kUmEpiThreads = 128;
+constexpr int kUmEpiWarps = 8;                     // two per quarter of tensor memory: even and odd chunks of rows
+constexpr int kUmEpiThreads = kUmEpiWarps * 32;
+constexpr int kUmThreads = 64 + kUmEpiThreads;
 constexpr int kUmChunk = 16;                       // rows the epilogue handles at a time
 constexpr int kUmExLd = kUmChunk + 1;
 constexpr int kUmMaxStages = 8;
@@ -71,7 +72,7 @@ struct UmmaShared {
 };
 
 inline size_t umma_smem_bytes(int RB, int n_stages) {
-  return (size_t)n_stages * um_stage_bytes(RB) + (size_t)kUmFeat * kUmExLd * 4 + sizeof(UmmaShared) + 1024;
+  return (size_t)n_stages * um_stage_bytes(RB) + (size_t)kUmEpiWarps * 32 * kUmExLd * 4 + sizeof(UmmaShared) + 1024;
 }
 inline int umma_stages_for(int RB, int max_smem_optin) {
   int s = kUmMaxStages;
@@ -162,6 +163,33 @@ __device__ __forceinline__ int ld_acquire(const int* p) {
   return v;
 }
 
+// apply_epilogue's EPI_QKV case with the pair already located (tensor t = q, k or v; head; index i
+// inside the half head): rotary embedding of q and k at the row's position, q to its buffer, k and v
+// into the cache.  Same operations in the same order.
+__device__ __forceinline__ void um_qkv_epilogue(const EpiParams& ep, int t, int head, int i, int m, float v0, float v1) {
+  const int pos = ld_act(ep.row_pos + m);
+  if (pos < 0) return;
+  const int hp = ep.head_dim >> 1;
+  if (t < 2) {
+    const float c = ep.rope_cos[(size_t)pos * hp + i];
+    const float s = ep.rope_sin[(size_t)pos * hp + i];
+    const float r0 = v0 * c - v1 * s;
+    const float r1 = v1 * c + v0 * s;
+    v0 = r0;
+    v1 = r1;
+  }
+  if (t == 0) {
+    float* q = ep.out + (size_t)m * ep.out_ld + head * ep.head_dim;
+    q[i] = v0;
+    q[i + hp] = v1;
+  } else {
+    __nv_bfloat16* base = reinterpret_cast<__nv_bfloat16*>(t == 1 ? ep.kcache : ep.vcache);
+    __nv_bfloat16* dst = base + (((size_t)ld_act(ep.row_seq + m) * ep.n_heads + head) * ep.max_seq + pos) * ep.head_dim;
+    dst[i] = __float2bfloat16_rn(v0);
+    dst[i + hp] = __float2bfloat16_rn(v1);
+  }
+}
+
 template <typename Pred>
 __device__ __forceinline__ bool um_wait(Pred pred, int* error, volatile int* s_abort, int code) {
   if (pred()) return true;
@@ -190,7 +218,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(um_smem_raw) + 1023) & ~(uintptr_t)1023);
   const int stage_bytes = um_stage_bytes(p.RB);
   float* ex = reinterpret_cast<float*>(smem + (size_t)p.n_stages * stage_bytes);
-  UmmaShared* sh = reinterpret_cast<UmmaShared*>(ex + kUmFeat * kUmExLd);
+  UmmaShared* sh = reinterpret_cast<UmmaShared*>(ex + kUmEpiWarps * 32 * kUmExLd);
   const int tid = threadIdx.x, warp = tid >> 5, lane = tid & 31;
   const int cta = blockIdx.x, n_cta = gridDim.x;
   const int KB = p.KB;
@@ -205,7 +233,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
     }
     for (int b = 0; b < 2; ++b) {
       mbar_init(&sh->acc_full[b], 1);
-      mbar_init(&sh->acc_empty[b], 4);
+      mbar_init(&sh->acc_empty[b], kUmEpiWarps);
     }
     sh->abort = *reinterpret_cast<volatile int*>(p.error) != 0 ? 1 : 0;  // an earlier kernel gave up: do nothing
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -336,8 +364,10 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
     }
   } else {
     // ================= epilogue: 4 warps, warp w reads lanes 32*(w%4).. of tensor memory =================
-    const int et = tid - 64;                 // 0..127
-    const int quarter = warp & 3;
+    const int et = tid - 64;                 // 0..255
+    const int ew = warp - 2;                 // epilogue warp 0..7
+    const int quarter = warp & 3;            // the quarter of tensor memory this warp may read (warp index mod 4)
+    const int chalf = ew >> 2;               // it takes the chunks of rows c = chalf, chalf + 2, ...
     const int R = quarter * 32 + lane;       // tile row (tensor-memory lane) of this thread
     const int pl = quarter * 16 + (lane & 15), half = lane >> 4;  // the output pair it finishes and which 8 rows of a chunk
     int buf = 0;
@@ -398,8 +428,18 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
       const int row0 = rb * RB;
       ensure_inv(rb);
       float* my_post = p.partial + (size_t)cta * (RB * kUmFeat);
-      for (int c = 0; c < RB / kUmChunk; ++c) {
-        if (row0 + c * kUmChunk >= p.M) break;  // rows that carry nothing (uniform)
+      // the output pair this thread finishes, located once per piece (not once per row)
+      const int pg = ft * 64 + pl;
+      int q_t = 0, q_head = 0, q_i = 0;
+      if (p.ep.mode == EPI_QKV) {
+        const int hp = p.ep.head_dim >> 1, per_tensor = p.ep.n_heads * hp;
+        q_t = pg / per_tensor;
+        const int rem = pg - q_t * per_tensor;
+        q_head = rem / hp;
+        q_i = rem - q_head * hp;
+      }
+      for (int c = chalf; c < RB / kUmChunk; c += 2) {
+        if (row0 + c * kUmChunk >= p.M) break;  // rows that carry nothing (uniform over the warp)
         float hi[16], lo[16];
         const uint32_t taddr = tmem_base + ((uint32_t)(quarter * 32) << 16) + (uint32_t)(buf * 2 * RB + c * kUmChunk);
         um_ld16(taddr, hi);
@@ -418,7 +458,6 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
         }
         // The two features of an output pair sit 16 lanes apart in the same warp: one shuffle per
         // row brings them together, and thread (pair, half) finishes rows half*8 .. half*8+7.
-        const int pg = ft * 64 + pl;
         const bool want_img = p.img_out != nullptr;
         float keep0[8], keep1[8];  // results this thread owes the output image
 #pragma unroll
@@ -446,6 +485,8 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
             } else if (p.ep.mode == EPI_SWIGLU && want_img) {
               keep0[t8] = (v0 / (1.0f + __expf(-v0))) * v1;
               if (p.ep.out != nullptr) p.ep.out[(size_t)m * p.ep.out_ld + pg] = keep0[t8];
+            } else if (p.ep.mode == EPI_QKV) {
+              um_qkv_epilogue(p.ep, q_t, q_head, q_i, m, v0, v1);
             } else {
               apply_epilogue<__nv_bfloat16>(p.ep, pg, m, v0, v1);
             }
@@ -456,7 +497,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
           // pieces of the image (8 consecutive features of one row, high parts and low parts).  A warp
           // covers 32 consecutive features of the residual stream, or 16 consecutive columns of u.
           const bool resid = p.ep.mode == EPI_RESID;
-          float* exw = ex + quarter * (32 * kUmExLd);
+          float* exw = ex + ew * (32 * kUmExLd);
           const int li = lane & 15;
           const int f0 = resid ? ((li >> 3) << 4) + (li & 7) : li;
           __syncwarp();
@@ -511,7 +552,6 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
       } else if (owner) {
         um_epi_sync();  // every thread has read the posts
         if (et < n_posts) p.flags[sh->posts[et]] = 0;
-        if (et + kUmEpiThreads < n_posts) p.flags[sh->posts[et + kUmEpiThreads]] = 0;
       }
       if ((buf ^= 1) == 0) acc_phase ^= 1u;
       u += s.kb1 - s.kb0;
