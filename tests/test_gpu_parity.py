@@ -729,3 +729,27 @@ def test_bf16_error_budget_against_unrounded_cache(tiny_bf16, l7b4, capsys):
             print("\n[bf16 error budget] %s: library vs oracle (K/V rounded on both sides) %.3e; library vs oracle with fp32 K/V %.3e; "
                   "the two oracles against each other %.3e" % (name, e_same, e_unr, e_kv))
         assert e_same < 1e-2 and e_unr < 1e-2
+
+
+def test_long_context_against_oracle():
+    """The 13B configuration's context length (2048-token prompt, keys up to ~2300) at the 7B layer
+    shapes, four layers deep: the prompt goes through the dense path in 16 row blocks, decode
+    attention walks 33+ chunks of 64 keys per head (4-5 per split), and every generated token is
+    checked against the oracle's recomputation of the whole sequence."""
+    shape = si.LLAMA7B_4L
+    plen, n_new = 2048, 40
+    eng, m, _ = make_pair(shape, (1, 2), max_seq=plen + n_new + 16, k_max=4, draw_device="cuda:0")
+    try:
+        prompt = si.make_prompts(shape.vocab, 1, plen, seed=96)
+        out = eng.sdfp_generate(prompt, 4, n_new)
+        ar = eng.sdfp_generate(prompt, 0, n_new)
+        assert out.tokens == ar.tokens
+        reported = check_stream_against_oracle(m, prompt[0].tolist(), out.tokens[0])
+        assert len(reported) <= 2, reported
+        # logits of three more positions through the decode kernels over the 2088-key cache
+        toks = prompt[0].tolist() + out.tokens[0]
+        got = eng.sdfp_forward_logits(toks[-3:], len(toks) - 3)
+        ref = orc.forward_nocache(m, toks).detach().numpy()[-3:]
+        assert max(rel_l2(got[r], ref[r]) for r in range(3)) < 1e-2
+    finally:
+        eng.close()
