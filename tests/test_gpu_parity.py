@@ -753,3 +753,21 @@ def test_long_context_against_oracle():
         assert max(rel_l2(got[r], ref[r]) for r in range(3)) < 1e-2
     finally:
         eng.close()
+
+
+def test_time_linear_hook_on_both_bf16_paths():
+    """The roofline hook of the linear kernels: per-operation mma.sync kernels (flag) and the tcgen05
+    kernel of a wide context; bytes are the matrix's, times are sane."""
+    shape = si.LLAMA7B_4L
+    d, f, v = shape.d_model, shape.d_ffn, shape.vocab
+    want = [3 * d * d * 2, d * d * 2, 2 * f * d * 2, d * f * 2, v * d * 2]
+    for kw in (dict(flags=pkg.FLAG_NO_PASS_KERNEL), dict(max_batch=8, k_max=4)):
+        eng, _, _ = make_pair(shape, (1, 2), max_seq=128, draw_device="cuda:0", **kw)
+        try:
+            for which in range(5):
+                ms, nbytes = eng.sdfp_time_linear(which, 8, 8)
+                assert nbytes == want[which] and 0.002 < ms < 5.0
+            with pytest.raises(pkg.SdfpError):
+                eng.sdfp_time_pass(False, 1, 0, 2)            # neither context runs the whole-pass kernel
+        finally:
+            eng.close()

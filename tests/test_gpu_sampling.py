@@ -142,3 +142,29 @@ def test_sampled_tokens_match_oracle_vocab_32000():
         assert 0 < accepted < drafted                  # both outcomes of the accept test occurred
     finally:
         eng.close()
+
+
+def test_sampled_decoding_on_the_dense_path():
+    """A bf16 context too wide for the whole-pass kernel (4 sequences x 5 rows) decodes on the tcgen05
+    path: sampled speculative decoding of a batch against the oracle, sequence by sequence (the
+    sequence index is part of the Philox counter), and the autoregressive sampler likewise."""
+    eng, m, _ = make_pair(si.TINY_BF16, (1, 2), max_seq=96, max_batch=4, k_max=4)
+    try:
+        prompts = si.make_prompts(m.vocab, 4, 20, seed=33)
+        T = 1.0 / 8.0
+        same = total = 0
+        for seed in range(6):
+            out = eng.sdfp_generate(prompts, 4, 16, temperature=T, seed=seed)
+            ar = eng.sdfp_generate(prompts, 0, 16, temperature=T, seed=seed)
+            for b in range(4):
+                ref = orc.spec_generate(orc.CachedLM(m, max_seq=96), orc.CachedLM(m, [0, 3], max_seq=96),
+                                        prompts[b].tolist(), 4, 16, temperature=T, seed=seed, seq=b)
+                ar_ref = orc.ar_generate(orc.CachedLM(m, max_seq=96), prompts[b].tolist(), 16, temperature=T, seed=seed, seq=b)
+                total += 2
+                same += (out.tokens[b] == ref.tokens) + (ar.tokens[b] == ar_ref.tokens)
+                if out.tokens[b] == ref.tokens:
+                    acc_b = [int(a) for a, d in zip(out.stats[:, b, 1], out.stats[:, b, 0]) if d > 0]
+                    assert acc_b == [r.accepted for r in ref.rounds]
+        assert same >= total - 3
+    finally:
+        eng.close()
