@@ -118,6 +118,7 @@ struct sdfp_ctx {
   bool dense_decode = false;       // ... this context's decode passes run on it as well
   void* um_lm_head = nullptr;
   unsigned char* um_x = nullptr;   // activation image, rows_cap (rounded to 128) x widest K
+  unsigned char *um_pa = nullptr, *um_pu = nullptr;  // prompt pass: images of the attention output and of u
   // decode on the dense path: images of gain * h, of the attention output and of u; sums of squares
   unsigned char *um_xh = nullptr, *um_xa = nullptr, *um_xu = nullptr;
   float* um_ssq = nullptr;
@@ -963,7 +964,9 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   if (c->use_dense) {
     const size_t rows128 = ((R + 127) / 128) * 128;
     const size_t kmax = (size_t)(((std::max(g.d_model, g.d_ffn) + kUmBK - 1) / kUmBK) * kUmBK);
-    if ((r = dev_alloc(c, &c->um_x, rows128 * kmax * 4, true)) ||
+    const size_t kd64 = (size_t)(((g.d_model + kUmBK - 1) / kUmBK) * kUmBK), kf64 = (size_t)(((g.d_ffn + kUmBK - 1) / kUmBK) * kUmBK);
+    if ((r = dev_alloc(c, &c->um_x, rows128 * kmax * 4, true)) || (r = dev_alloc(c, &c->um_pa, rows128 * kd64 * 4, true)) ||
+        (r = dev_alloc(c, &c->um_pu, rows128 * kf64 * 4, true)) ||
         (r = dev_alloc(c, &c->um_partial, (size_t)c->num_sms * kUmMaxRB * kUmFeat)) ||
         (r = dev_alloc(c, &c->um_flags, (size_t)c->num_sms, true)) || (r = dev_alloc(c, &c->um_error, 1, true)) ||
         (r = dev_alloc(c, &c->h_fork, R * g.d_model)))
@@ -1138,35 +1141,49 @@ int prefill_range(sdfp_ctx* c, bool draft, int b, int from, int to) {
 // pruned layer see the same tokens through the same weights, so their K/V ARE the target's.  The
 // target's pass leaves the residual rows at that point in `h_fork`; the draft copies the K/V of
 // those layers and runs only the kept layers behind the fork.
+// gate/up + SwiGLU, whose epilogue leaves u as the operand image of the down-projection, then down + residual
+int dense_ffn_block(sdfp_ctx* c, const LayerWeights& lw, int rows, int RB, int KBf) {
+  const int d = c->cfg.d_model, f = c->cfg.d_ffn;
+  const int KBd = (d + kUmBK - 1) / kUmBK;
+  CU_OK(c, launch(c, prep_rows_kernel, dim3((rows + 7) / 8), dim3(kPrepThreads), 0, (const float*)c->h, d, rows, d,
+                  (const float*)lw.ffn_gain, c->cfg.rms_eps, c->um_x, RB, KBd));
+  UmmaParams gu = dense_params(c, lw.um_gu, c->um_x, rows, RB, KBd, f, base_epi(c, EPI_SWIGLU, nullptr, f));
+  gu.img_out = c->um_pu;
+  gu.img_KB = KBf;
+  CU_OK(c, launch_dense(c, gu));
+  CU_OK(c, launch_dense(c, dense_params(c, lw.um_down, c->um_pu, rows, RB, KBf, d / 2, base_epi(c, EPI_RESID, c->h, d))));
+  return 0;
+}
+
 int dense_layer(sdfp_ctx* c, const KvCache& kv, int l, int b, int rows, bool run_attn, bool run_ffn) {
   const sdfp_config& g = c->cfg;
   const int d = g.d_model, f = g.d_ffn;
   const LayerWeights& lw = c->layers[l];
   if (run_ffn && !run_attn) {
-    CU_OK(c, run_dense_linear(c, lw.um_gu, c->h, d, rows, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
-    CU_OK(c, run_dense_linear(c, lw.um_down, c->u, f, rows, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
-    return 0;
+    const int RB0 = rows >= kUmMaxRB ? kUmMaxRB : ((rows + 15) / 16) * 16;
+    return dense_ffn_block(c, lw, rows, RB0, (f + kUmBK - 1) / kUmBK);
   }
   if (!run_attn) return 0;
+  const int RB = rows >= kUmMaxRB ? kUmMaxRB : ((rows + 15) / 16) * 16;  // as run_dense_linear chooses it
+  const int KBd = (d + kUmBK - 1) / kUmBK, KBf = (f + kUmBK - 1) / kUmBK;
   EpiParams qkv = base_epi(c, EPI_QKV, c->q, d);
   qkv.kcache = kv.k[l];
   qkv.vcache = kv.v[l];
   CU_OK(c, run_dense_linear(c, lw.um_qkv, c->h, d, rows, d, 3 * d / 2, lw.attn_gain, qkv));
+  // the attention output and the SwiGLU output are written as operand images by their producers
   const float scale = 1.0f / std::sqrt((float)g.head_dim);
   const dim3 grid((rows + kPfaQ - 1) / kPfaQ, g.n_heads);
   const __nv_bfloat16* kc = reinterpret_cast<const __nv_bfloat16*>(kv.k[l]);
   const __nv_bfloat16* vc = reinterpret_cast<const __nv_bfloat16*>(kv.v[l]);
   if (g.head_dim == 128)
     CU_OK(c, launch(c, prefill_attention_kernel<128>, grid, dim3(kPfaThreads), prefill_attention_smem<128>(), (const float*)c->q, kc,
-                    vc, c->att, rows, g.n_heads, g.max_seq, b, scale));
+                    vc, c->att, rows, g.n_heads, g.max_seq, b, scale, c->um_pa, RB, KBd));
   else
     CU_OK(c, launch(c, prefill_attention_kernel<64>, grid, dim3(kPfaThreads), prefill_attention_smem<64>(), (const float*)c->q, kc, vc,
-                    c->att, rows, g.n_heads, g.max_seq, b, scale));
-  CU_OK(c, run_dense_linear(c, lw.um_wo, c->att, d, rows, d, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
+                    c->att, rows, g.n_heads, g.max_seq, b, scale, c->um_pa, RB, KBd));
+  CU_OK(c, launch_dense(c, dense_params(c, lw.um_wo, c->um_pa, rows, RB, KBd, d / 2, base_epi(c, EPI_RESID, c->h, d))));
   if (!run_ffn) return 0;
-  CU_OK(c, run_dense_linear(c, lw.um_gu, c->h, d, rows, d, f, lw.ffn_gain, base_epi(c, EPI_SWIGLU, c->u, f)));
-  CU_OK(c, run_dense_linear(c, lw.um_down, c->u, f, rows, f, d / 2, nullptr, base_epi(c, EPI_RESID, c->h, d)));
-  return 0;
+  return dense_ffn_block(c, lw, rows, RB, KBf);
 }
 
 int first_pruned_layer(const sdfp_ctx* c) {

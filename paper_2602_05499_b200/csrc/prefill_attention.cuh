@@ -51,7 +51,7 @@ template <int HD>
 __global__ void __launch_bounds__(kPfaThreads)
 prefill_attention_kernel(const float* __restrict__ q, const __nv_bfloat16* __restrict__ kcache,
                          const __nv_bfloat16* __restrict__ vcache, float* __restrict__ out, int M, int n_heads, int max_seq,
-                         int seq, float scale) {
+                         int seq, float scale, unsigned char* __restrict__ img, int img_rb, int img_kb) {
   constexpr int LD = HD + 8;
   extern __shared__ __align__(16) unsigned char pfa_smem[];
   __nv_bfloat16* sQh = reinterpret_cast<__nv_bfloat16*>(pfa_smem);
@@ -210,11 +210,27 @@ prefill_attention_kernel(const float* __restrict__ q, const __nv_bfloat16* __res
     l_run[r] += __shfl_xor_sync(0xffffffffu, l_run[r], 2);
   }
   const float inv_a = 1.0f / l_run[0], inv_b = 1.0f / l_run[1];
+  // The result goes out as fp32 rows, or (img non-null) straight into the activation image of the
+  // O-projection on the dense path: bf16 hi + lo, two neighbouring columns per 4-byte store (layout
+  // as in attn_store of attention.cuh: row block img_rb, img_kb k blocks of 64).
+  auto put = [&](int m, int col, float x0, float x1) {
+    if (img == nullptr) {
+      *reinterpret_cast<float2*>(out + (size_t)m * d_model + col) = make_float2(x0, x1);
+      return;
+    }
+    const int rb = m / img_rb, tm = m - rb * img_rb, kg = col >> 3;
+    unsigned char* p = img + ((size_t)rb * img_kb + (kg >> 3)) * ((size_t)img_rb * 256) + (size_t)(kg & 7) * (img_rb * 32) +
+                       (size_t)(tm >> 3) * 128 + (tm & 7) * 16 + (col & 7) * 2;
+    uint32_t hi, lo;
+    split_pack(x0, x1, hi, lo);
+    *reinterpret_cast<uint32_t*>(p) = hi;
+    *reinterpret_cast<uint32_t*>(p + (size_t)img_rb * 16) = lo;
+  };
 #pragma unroll
   for (int j = 0; j < HD / 8; ++j) {
     const int d = j * 8 + 2 * qd;
-    if (row_a < M) *reinterpret_cast<float2*>(out + (size_t)row_a * d_model + head * HD + d) = make_float2(o[j][0] * inv_a, o[j][1] * inv_a);
-    if (row_b < M) *reinterpret_cast<float2*>(out + (size_t)row_b * d_model + head * HD + d) = make_float2(o[j][2] * inv_b, o[j][3] * inv_b);
+    if (row_a < M) put(row_a, head * HD + d, o[j][0] * inv_a, o[j][1] * inv_a);
+    if (row_b < M) put(row_b, head * HD + d, o[j][2] * inv_b, o[j][3] * inv_b);
   }
 }
 

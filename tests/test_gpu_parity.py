@@ -771,3 +771,20 @@ def test_time_linear_hook_on_both_bf16_paths():
                 eng.sdfp_time_pass(False, 1, 0, 2)            # neither context runs the whole-pass kernel
         finally:
             eng.close()
+
+
+def test_largest_batch_and_row_count():
+    """The library's limits in one context: 16 sequences, k = 4, 80 rows in a verify pass (row block of
+    80 rows = MMA width 160), 32 rows in the first draft pass; prompts of one token (nothing to cache
+    before the first round).  Speculative == autoregressive, sequences independent."""
+    eng, m, _ = make_pair(si.TINY_BF16, (1, 2), max_seq=64, max_batch=16, k_max=4)
+    try:
+        for plen in (1, 9):
+            prompts = si.make_prompts(m.vocab, 16, plen, seed=97)
+            out = eng.sdfp_generate(prompts, 4, 20)
+            assert out.tokens == eng.sdfp_generate(prompts, 0, 20).tokens
+            for b in (0, 7, 15):
+                assert eng.sdfp_generate(prompts[b:b + 1], 4, 20).tokens[0] == out.tokens[b]
+                check_stream_against_oracle(m, prompts[b].tolist(), out.tokens[b])
+    finally:
+        eng.close()
