@@ -116,6 +116,7 @@ struct sdfp_ctx {
   // a context whose widest pass does not fit the whole-pass kernel
   bool use_dense = false;
   bool dense_decode = false;       // ... this context's decode passes run on it as well
+  int attn_splits = 1;             // its attention kernel: CTAs per (sequence, head), fixed for the life of the context
   void* um_lm_head = nullptr;
   unsigned char* um_x = nullptr;   // activation image, rows_cap (rounded to 128) x widest K
   unsigned char *um_pa = nullptr, *um_pu = nullptr;  // prompt pass: images of the attention output and of u
@@ -297,20 +298,26 @@ cudaError_t run_attention(sdfp_ctx* c, const KvCache& kv, int layer, int rows, i
   ap.scale = 1.0f / std::sqrt((float)c->cfg.head_dim);
   const int n_groups = rows / rows_per_seq;
   const bool hd128 = c->cfg.head_dim == 128;
-  if (c->dense_decode) {  // a fixed number of splits per (sequence, head), each walking its chunks
-    const dim3 grid(kAttnSplits, ap.n_heads, n_groups);
-    const dim3 block(kHalfThreads);
+  if (c->dense_decode) {
+    // streaming kernel: row capacity 2 (draft and autoregressive passes), 5 (verify at k <= 4) or 8
+    // (wider row counts run as groups of 8 rows)
+    ap.n_splits = c->attn_splits;
+    ap.error = c->um_error;
+    ap.zero = 0u;
     const int R = rows_per_seq;
+    const dim3 block(kAsThreads);
+    auto go = [&](auto kernel, int rm, size_t sm) {
+      const dim3 grid(ap.n_splits, ap.n_heads, n_groups * ((R + rm - 1) / rm));
+      return launch(c, kernel, grid, block, sm, ap, rows);
+    };
     if (hd128) {
-      const size_t sm = pass_attn_smem_half<128>();
-      if (R <= 2) return launch(c, attention_split_kernel<128, 2>, grid, block, sm, ap, rows);
-      if (R <= 8) return launch(c, attention_split_kernel<128, 8>, grid, block, sm, ap, rows);
-      return launch(c, attention_split_kernel<128, 16>, grid, block, sm, ap, rows);
+      if (R <= 2) return go(attention_stream_kernel<128, 2, 8>, 2, attention_stream_smem<128, 2>());
+      if (R <= 5) return go(attention_stream_kernel<128, 5, 8>, 5, attention_stream_smem<128, 5>());
+      return go(attention_stream_kernel<128, 8, 8>, 8, attention_stream_smem<128, 8>());
     }
-    const size_t sm = pass_attn_smem_half<64>();
-    if (R <= 2) return launch(c, attention_split_kernel<64, 2>, grid, block, sm, ap, rows);
-    if (R <= 8) return launch(c, attention_split_kernel<64, 8>, grid, block, sm, ap, rows);
-    return launch(c, attention_split_kernel<64, 16>, grid, block, sm, ap, rows);
+    if (R <= 2) return go(attention_stream_kernel<64, 2, 8>, 2, attention_stream_smem<64, 2>());
+    if (R <= 5) return go(attention_stream_kernel<64, 5, 8>, 5, attention_stream_smem<64, 5>());
+    return go(attention_stream_kernel<64, 8, 8>, 8, attention_stream_smem<64, 8>());
   }
   if (c->bf16)
     return hd128 ? launch_attention_t<__nv_bfloat16, 128>(c, ap, n_groups)
@@ -908,6 +915,26 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
       return bail(SDFP_ECUDA);
     }
   }
+  if (c->dense_decode) {
+    // As many splits as still give one wave of CTAs (two per SM) when every sequence slot is in
+    // use: more CTAs than that only add set-up and fold time (7B shape, batch 8, context ~600: 21 / 27
+    // / 33 / 44 us per layer at 1 / 2 / 4 / 8 splits).  One number for all passes of the context,
+    // because the order in which a row's keys are added depends on it.
+    c->attn_splits = std::min((int)kAttnSplits, std::max(1, 2 * c->num_sms / (g.max_batch * g.n_heads)));
+    auto cfg_attn = [](auto kernel, size_t sm) {
+      return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) == cudaSuccess;
+    };
+    const bool ok = g.head_dim == 128 ? (cfg_attn(attention_stream_kernel<128, 2, 8>, attention_stream_smem<128, 2>()) &&
+                                         cfg_attn(attention_stream_kernel<128, 5, 8>, attention_stream_smem<128, 5>()) &&
+                                         cfg_attn(attention_stream_kernel<128, 8, 8>, attention_stream_smem<128, 8>()))
+                                      : (cfg_attn(attention_stream_kernel<64, 2, 8>, attention_stream_smem<64, 2>()) &&
+                                         cfg_attn(attention_stream_kernel<64, 5, 8>, attention_stream_smem<64, 5>()) &&
+                                         cfg_attn(attention_stream_kernel<64, 8, 8>, attention_stream_smem<64, 8>()));
+    if (!ok) {
+      c->err = "dense-path attention kernel configuration failed";
+      return bail(SDFP_ECUDA);
+    }
+  }
   if (c->use_pass) {
     const cudaError_t pe = g.head_dim == 128 ? configure_pass_t<128>(c, optin) : configure_pass_t<64>(c, optin);
     if (pe != cudaSuccess) {
@@ -1059,9 +1086,10 @@ int check_dense_error(sdfp_ctx* c) {
   cudaMemsetAsync(c->um_flags, 0, (size_t)c->num_sms * sizeof(int), c->stream);
   cudaStreamSynchronize(c->stream);
   static const char* const what[] = {"", "pipeline stage never freed", "pipeline stage never filled", "accumulator never freed",
-                                     "accumulator never finished", "partial accumulator of a cut tile never posted"};
-  return fail(c, SDFP_ETIMEOUT, "dense linear kernel gave up a wait (%s); results of this call are invalid",
-              e >= 1 && e <= 5 ? what[e] : "unknown");
+                                     "accumulator never finished", "partial accumulator of a cut tile never posted",
+                                     "K/V stage of the attention kernel never filled", "K/V stage of the attention kernel never freed"};
+  return fail(c, SDFP_ETIMEOUT, "a kernel of the dense path gave up a wait (%s); results of this call are invalid",
+              e >= 1 && e <= 7 ? what[e] : "unknown");
 }
 
 // A failed wait inside the pass kernel leaves its code in device memory; turn it into an error
