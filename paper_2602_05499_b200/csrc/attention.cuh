@@ -38,11 +38,8 @@ struct AttnParams {
   // (m % rb / 8) * 128 + (m % 8) * 16, low parts rb * 16 bytes further)
   unsigned char* img;
   int img_rb, img_kb;
-  // streaming kernel of the dense path only: splits per (sequence, head), the dense path's error
-  // word for waits that run out, and a zero the compiler cannot see
+  // dense path only: CTAs per (sequence, head), each taking every n_splits-th 64-key chunk
   int n_splits;
-  int* error;
-  unsigned zero;
 };
 
 __device__ __forceinline__ void attn_store(const AttnParams& ap, float* dst, int m, int col, float v) {

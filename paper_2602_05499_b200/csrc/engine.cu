@@ -299,25 +299,10 @@ cudaError_t run_attention(sdfp_ctx* c, const KvCache& kv, int layer, int rows, i
   const int n_groups = rows / rows_per_seq;
   const bool hd128 = c->cfg.head_dim == 128;
   if (c->dense_decode) {
-    // streaming kernel: row capacity 2 (draft and autoregressive passes), 5 (verify at k <= 4) or 8
-    // (wider row counts run as groups of 8 rows)
     ap.n_splits = c->attn_splits;
-    ap.error = c->um_error;
-    ap.zero = 0u;
-    const int R = rows_per_seq;
-    const dim3 block(kAsThreads);
-    auto go = [&](auto kernel, int rm, size_t sm) {
-      const dim3 grid(ap.n_splits, ap.n_heads, n_groups * ((R + rm - 1) / rm));
-      return launch(c, kernel, grid, block, sm, ap, rows);
-    };
-    if (hd128) {
-      if (R <= 2) return go(attention_stream_kernel<128, 2, 8>, 2, attention_stream_smem<128, 2>());
-      if (R <= 5) return go(attention_stream_kernel<128, 5, 8>, 5, attention_stream_smem<128, 5>());
-      return go(attention_stream_kernel<128, 8, 8>, 8, attention_stream_smem<128, 8>());
-    }
-    if (R <= 2) return go(attention_stream_kernel<64, 2, 8>, 2, attention_stream_smem<64, 2>());
-    if (R <= 5) return go(attention_stream_kernel<64, 5, 8>, 5, attention_stream_smem<64, 5>());
-    return go(attention_stream_kernel<64, 8, 8>, 8, attention_stream_smem<64, 8>());
+    const dim3 grid(ap.n_splits, ap.n_heads, n_groups);
+    if (hd128) return launch(c, attention_mma_kernel<128>, grid, dim3(kAmThreads), attention_mma_smem<128>(), ap, rows);
+    return launch(c, attention_mma_kernel<64>, grid, dim3(kAmThreads), attention_mma_smem<64>(), ap, rows);
   }
   if (c->bf16)
     return hd128 ? launch_attention_t<__nv_bfloat16, 128>(c, ap, n_groups)
@@ -917,19 +902,15 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
   }
   if (c->dense_decode) {
     // As many splits as still give one wave of CTAs (two per SM) when every sequence slot is in
-    // use: more CTAs than that only add set-up and fold time (7B shape, batch 8, context ~600: 21 / 27
-    // / 33 / 44 us per layer at 1 / 2 / 4 / 8 splits).  One number for all passes of the context,
+    // use: more CTAs than that only add set-up and fold time (7B shape, batch 8, context ~600: 4.11 /
+    // 4.34 / 4.61 ms per 8-row pass at 1 / 2 / 4 splits).  One number for all passes of the context,
     // because the order in which a row's keys are added depends on it.
     c->attn_splits = std::min((int)kAttnSplits, std::max(1, 2 * c->num_sms / (g.max_batch * g.n_heads)));
     auto cfg_attn = [](auto kernel, size_t sm) {
       return cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)sm) == cudaSuccess;
     };
-    const bool ok = g.head_dim == 128 ? (cfg_attn(attention_stream_kernel<128, 2, 8>, attention_stream_smem<128, 2>()) &&
-                                         cfg_attn(attention_stream_kernel<128, 5, 8>, attention_stream_smem<128, 5>()) &&
-                                         cfg_attn(attention_stream_kernel<128, 8, 8>, attention_stream_smem<128, 8>()))
-                                      : (cfg_attn(attention_stream_kernel<64, 2, 8>, attention_stream_smem<64, 2>()) &&
-                                         cfg_attn(attention_stream_kernel<64, 5, 8>, attention_stream_smem<64, 5>()) &&
-                                         cfg_attn(attention_stream_kernel<64, 8, 8>, attention_stream_smem<64, 8>()));
+    const bool ok = g.head_dim == 128 ? cfg_attn(attention_mma_kernel<128>, attention_mma_smem<128>())
+                                       : cfg_attn(attention_mma_kernel<64>, attention_mma_smem<64>());
     if (!ok) {
       c->err = "dense-path attention kernel configuration failed";
       return bail(SDFP_ECUDA);
@@ -1086,10 +1067,9 @@ int check_dense_error(sdfp_ctx* c) {
   cudaMemsetAsync(c->um_flags, 0, (size_t)c->num_sms * sizeof(int), c->stream);
   cudaStreamSynchronize(c->stream);
   static const char* const what[] = {"", "pipeline stage never freed", "pipeline stage never filled", "accumulator never freed",
-                                     "accumulator never finished", "partial accumulator of a cut tile never posted",
-                                     "K/V stage of the attention kernel never filled", "K/V stage of the attention kernel never freed"};
-  return fail(c, SDFP_ETIMEOUT, "a kernel of the dense path gave up a wait (%s); results of this call are invalid",
-              e >= 1 && e <= 7 ? what[e] : "unknown");
+                                     "accumulator never finished", "partial accumulator of a cut tile never posted"};
+  return fail(c, SDFP_ETIMEOUT, "dense linear kernel gave up a wait (%s); results of this call are invalid",
+              e >= 1 && e <= 5 ? what[e] : "unknown");
 }
 
 // A failed wait inside the pass kernel leaves its code in device memory; turn it into an error
