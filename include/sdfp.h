@@ -289,13 +289,18 @@ int sdfp_time_pass(sdfp_ctx *ctx, int32_t draft, int32_t rows, int32_t position,
                    float *ms_per_launch, int64_t *bytes_per_launch);
 
 /*
- * Failure-path test hook (whole-pass kernel contexts; SDFP_ESTATE otherwise).  Section II-A's
- * loop has no counterpart: this exercises the library's own bounded waits.  After the call,
- * the grid barriers of the next pass expect one arrival more than the grid can provide and
- * every wait gives up after wait_limit_ns (1 ms .. 2 s) instead of the default 2 s: that pass
- * winds down in an orderly way (nothing faults, nothing spins on), the entry point that
- * launched it returns SDFP_ETIMEOUT with the name of the wait in sdfp_last_error, and in
- * doing so puts barrier and limit back to normal, so the next call on the context works.
+ * Failure-path test hook (bf16 contexts whose passes run in the whole-pass kernel or on the
+ * dense path; SDFP_ESTATE otherwise).  Section II-A's loop has no counterpart: this exercises
+ * the library's own bounded waits.  Whole-pass kernel: after the call, the grid barriers of the
+ * next pass expect one arrival more than the grid can provide.  Dense path: in the next
+ * sdfp_forward_logits or sdfp_forward_logits_static call (other entry points are not affected),
+ * the CTAs of the linear kernels that hold the middle of a feature tile raise their "partial
+ * sum posted" flags where nobody looks, so the CTA that finishes the tile waits for a post that
+ * never comes.  Either way every wait gives up after wait_limit_ns (1 ms .. 2 s) instead of
+ * the default 2 s: that pass winds down in an orderly way (nothing faults, nothing spins on),
+ * the entry point that launched it returns SDFP_ETIMEOUT with the name of the wait in
+ * sdfp_last_error, and in doing so puts everything back to normal, so the next call on the
+ * context works.
  */
 int sdfp_debug_expire_next_wait(sdfp_ctx *ctx, uint64_t wait_limit_ns);
 

@@ -125,6 +125,9 @@ struct sdfp_ctx {
   float* um_ssq = nullptr;
   float* um_partial = nullptr;
   int *um_flags = nullptr, *um_error = nullptr;
+  int* um_flags_dummy = nullptr;          // failure-path test hook: where posts go to be lost
+  unsigned long long um_expire_ns = 0;    // hook armed: the next sdfp_forward_logits call runs with ...
+  unsigned long long um_sabotage_ns = 0;  // ... lost posts and this wait limit
   int rows_cap = kMaxRows;         // rows the activation buffers h, q, att, u and the row plan hold
   int max_smem_optin = 0;
   bool own_stream = false;
@@ -213,7 +216,9 @@ UmmaParams dense_params(const sdfp_ctx* c, const void* w_img, const unsigned cha
   p.n_stages = umma_stages_for(RB, c->max_smem_optin);
   p.partial = c->um_partial;
   p.flags = c->um_flags;
+  p.flags_post = c->um_sabotage_ns ? c->um_flags_dummy : c->um_flags;  // test hook: posts that never arrive
   p.error = c->um_error;
+  p.wait_limit_ns = c->um_sabotage_ns ? c->um_sabotage_ns : kWaitLimitNs;
   p.ssq_ld = kMaxRows;
   p.inv_k = 1.0f;
   p.eps = c->cfg.rms_eps;
@@ -977,6 +982,7 @@ extern "C" int sdfp_create(const sdfp_config* cfg, const sdfp_weights* w, void* 
         (r = dev_alloc(c, &c->um_pu, rows128 * kf64 * 4, true)) ||
         (r = dev_alloc(c, &c->um_partial, (size_t)c->num_sms * kUmMaxRB * kUmFeat)) ||
         (r = dev_alloc(c, &c->um_flags, (size_t)c->num_sms, true)) || (r = dev_alloc(c, &c->um_error, 1, true)) ||
+        (r = dev_alloc(c, &c->um_flags_dummy, (size_t)c->num_sms, true)) ||
         (r = dev_alloc(c, &c->h_fork, R * g.d_model)))
       return bail(r);
     if (c->dense_decode) {
@@ -1065,6 +1071,7 @@ int check_dense_error(sdfp_ctx* c) {
   if (e == 0) return 0;
   cudaMemsetAsync(c->um_error, 0, sizeof(int), c->stream);
   cudaMemsetAsync(c->um_flags, 0, (size_t)c->num_sms * sizeof(int), c->stream);
+  cudaMemsetAsync(c->um_flags_dummy, 0, (size_t)c->num_sms * sizeof(int), c->stream);
   cudaStreamSynchronize(c->stream);
   static const char* const what[] = {"", "pipeline stage never freed", "pipeline stage never filled", "accumulator never freed",
                                      "accumulator never finished", "partial accumulator of a cut tile never posted"};
@@ -1091,7 +1098,18 @@ int check_pass_error(sdfp_ctx* c) {
 
 // Logits of `rows` tokens of sequence slot 0 at positions start.., in passes of as many rows as
 // one pass carries, so that a row's logits never depend on how many rows the caller asked for.
+int forward_logits_passes_inner(sdfp_ctx* c, bool draft, const int32_t* tokens, int rows, int start, float* host_logits);
+
+// (the failure-path test hook of the dense path applies to exactly one call of this function)
 int forward_logits_passes(sdfp_ctx* c, bool draft, const int32_t* tokens, int rows, int start, float* host_logits) {
+  c->um_sabotage_ns = c->um_expire_ns;
+  c->um_expire_ns = 0;
+  const int r = forward_logits_passes_inner(c, draft, tokens, rows, start, host_logits);
+  c->um_sabotage_ns = 0;
+  return r;
+}
+
+int forward_logits_passes_inner(sdfp_ctx* c, bool draft, const int32_t* tokens, int rows, int start, float* host_logits) {
   const sdfp_config& g = c->cfg;
   CU_OK(c, cudaMemcpyAsync(c->fwd_tok, tokens, (size_t)rows * 4, cudaMemcpyHostToDevice, c->stream));
   const int per_pass = c->use_pass ? kPassMaxRows : kMaxRows;
@@ -1481,9 +1499,14 @@ extern "C" int sdfp_forward_logits_static(sdfp_ctx* c, int32_t draft, const int3
 extern "C" int sdfp_debug_expire_next_wait(sdfp_ctx* c, uint64_t wait_limit_ns) {
   if (!c) return SDFP_EINVAL;
   if (int r = check_device(c, "sdfp_debug_expire_next_wait")) return r;
-  if (!c->use_pass) return fail(c, SDFP_ESTATE, "sdfp_debug_expire_next_wait: this context does not use the whole-pass kernel");
+  if (!c->use_pass && !c->dense_decode)
+    return fail(c, SDFP_ESTATE, "sdfp_debug_expire_next_wait: this context uses neither the whole-pass kernel nor the dense path for its passes");
   if (wait_limit_ns < 1000000ull || wait_limit_ns > 2000000000ull)
     return fail(c, SDFP_EINVAL, "sdfp_debug_expire_next_wait: the limit must lie between 1 ms and 2 s");
+  if (c->dense_decode) {  // the next sdfp_forward_logits[_static] call: see forward_logits_passes
+    c->um_expire_ns = wait_limit_ns;
+    return 0;
+  }
   const unsigned long long words[2] = {1ull, (unsigned long long)wait_limit_ns};  // bar_extra, wait_limit_ns
   CU_OK(c, cudaMemcpyAsync(&c->psync->bar_extra, words, sizeof words, cudaMemcpyHostToDevice, c->stream));
   CU_OK(c, cudaStreamSynchronize(c->stream));  // words is a local

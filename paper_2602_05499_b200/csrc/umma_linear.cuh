@@ -88,8 +88,10 @@ struct UmmaParams {
   int n_pairs;             // valid output pairs (<= 64 * n_ft)
   int n_stages;
   float* partial;          // [grid][RB * 128] partial accumulators of cut tiles
-  int* flags;              // [grid], zero between launches
+  int* flags;              // [grid], zero between launches: "CTA c has posted its partial accumulator"
+  int* flags_post;         // where a CTA raises its flag: flags, except under the failure-path test hook
   int* error;              // first UmmaError seen, sticky
+  unsigned long long wait_limit_ns;  // after this long a wait gives up (kWaitLimitNs unless the test hook shortens it)
   // RMSNorm folded in: the activation image carries gain * h; 1/rms of row m comes from ssq_groups
   // partial sums of squares ssq_in[g * ssq_ld + m] left by whoever wrote h (null: no norm)
   const float* ssq_in;
@@ -191,7 +193,7 @@ __device__ __forceinline__ void um_qkv_epilogue(const EpiParams& ep, int t, int 
 }
 
 template <typename Pred>
-__device__ __forceinline__ bool um_wait(Pred pred, int* error, volatile int* s_abort, int code) {
+__device__ __forceinline__ bool um_wait(Pred pred, int* error, volatile int* s_abort, int code, unsigned long long limit_ns) {
   if (pred()) return true;
   const unsigned long long t0 = global_ns();
   unsigned spins = 0;
@@ -199,7 +201,7 @@ __device__ __forceinline__ bool um_wait(Pred pred, int* error, volatile int* s_a
     if (pred()) return true;
     if (((++spins) & 63u) == 0) {
       if (*s_abort) return false;
-      if (global_ns() - t0 > kWaitLimitNs) {
+      if (global_ns() - t0 > limit_ns) {
         atomicCAS(error, 0, code);
         *s_abort = 1;
         return false;
@@ -294,7 +296,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
             } else if (early) {
               bulk_load(dst + kUmABytes, xsrc, (unsigned)um_b_stage_bytes(p.RB), &sh->full[stage], pol_x);
             } else {
-              ok = um_wait([&] { return mbar_try_wait(&sh->empty[stage], phase ^ 1u); }, p.error, s_abort, UMMA_ERR_STAGE_EMPTY);
+              ok = um_wait([&] { return mbar_try_wait(&sh->empty[stage], phase ^ 1u); }, p.error, s_abort, UMMA_ERR_STAGE_EMPTY, p.wait_limit_ns);
               if (!ok) break;
               mbar_arrive_expect_tx(&sh->full[stage], (unsigned)stage_bytes);
               bulk_load(dst, wsrc, kUmABytes, &sh->full[stage], pol);
@@ -320,7 +322,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
           const unsigned sl = j % (unsigned)p.n_stages, par = (j / (unsigned)p.n_stages) & 1u;
           const unsigned long long t0 = global_ns();
           while (!mbar_try_wait(&sh->full[sl], par))
-            if (global_ns() - t0 > kWaitLimitNs) break;
+            if (global_ns() - t0 > p.wait_limit_ns) break;
         }
       }
     }
@@ -334,12 +336,12 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
       bool ok = true;
       for (long long u = ub; u < ue && ok;) {
         const UmSeg s = next_seg(u);
-        ok = um_wait([&] { return mbar_try_wait(&sh->acc_empty[buf], acc_phase ^ 1u); }, p.error, s_abort, UMMA_ERR_ACC_EMPTY);
+        ok = um_wait([&] { return mbar_try_wait(&sh->acc_empty[buf], acc_phase ^ 1u); }, p.error, s_abort, UMMA_ERR_ACC_EMPTY, p.wait_limit_ns);
         if (!ok) break;
         um_fence_after();
         const uint32_t tmem_d = tmem_base + (uint32_t)(buf * 2 * p.RB);
         for (int kb = s.kb0; kb < s.kb1; ++kb) {
-          ok = um_wait([&] { return mbar_try_wait(&sh->full[stage], phase); }, p.error, s_abort, UMMA_ERR_STAGE_FULL);
+          ok = um_wait([&] { return mbar_try_wait(&sh->full[stage], phase); }, p.error, s_abort, UMMA_ERR_STAGE_FULL, p.wait_limit_ns);
           if (!ok) break;
           um_fence_after();
           const uint32_t a0 = smem_u32(smem + (size_t)stage * stage_bytes);
@@ -402,7 +404,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
       const int ft = s.tile / p.n_rb, rb = s.tile - ft * p.n_rb;
       const bool starts = s.kb0 == 0, whole = starts && s.kb1 == KB;
       const bool owner = starts && !whole;
-      const bool okw = um_wait([&] { return mbar_try_wait(&sh->acc_full[buf], acc_phase); }, p.error, s_abort, UMMA_ERR_ACC_FULL);
+      const bool okw = um_wait([&] { return mbar_try_wait(&sh->acc_full[buf], acc_phase); }, p.error, s_abort, UMMA_ERR_ACC_FULL, p.wait_limit_ns);
       (void)okw;
       if (owner && et == 0) {
         // the rest of the tile lies at the start of the ranges of the CTAs that follow
@@ -413,7 +415,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
           unit_range(n_units, c2, n_cta, b2, e2);
           if (b2 >= tile_end) break;
           if (e2 > b2) {
-            um_wait([&] { return ld_acquire(p.flags + c2) != 0; }, p.error, s_abort, UMMA_ERR_POST);
+            um_wait([&] { return ld_acquire(p.flags + c2) != 0; }, p.error, s_abort, UMMA_ERR_POST, p.wait_limit_ns);
             sh->posts[n++] = c2;
           }
         }
@@ -548,7 +550,7 @@ __global__ void __launch_bounds__(kUmThreads, 1) umma_linear_kernel(UmmaParams p
       if (!starts) {
         __threadfence();
         um_epi_sync();
-        if (et == 0) st_release(p.flags + cta, 1);
+        if (et == 0) st_release(p.flags_post + cta, 1);
       } else if (owner) {
         um_epi_sync();  // every thread has read the posts
         if (et < n_posts) p.flags[sh->posts[et]] = 0;

@@ -471,6 +471,32 @@ def test_wide_batch_7b_shape():
         eng.close()
 
 
+def test_dense_path_long_context():
+    """Decode attention of the dense path over many 64-key chunks (the ring of K/V tiles wraps, one
+    split per (sequence, head) walks every chunk) and chains of linear layers behind it: contexts of
+    300 to 330 keys at the 7B layer shapes, two sequences of an 8-slot context."""
+    shape = si.LLAMA7B_4L
+    eng, m, _ = make_pair(shape, (1, 2), max_seq=384, max_batch=8, k_max=4, draw_device="cuda:0")
+    try:
+        prompts = si.make_prompts(shape.vocab, 2, 300, seed=62)
+        out = eng.sdfp_generate(prompts, 4, 24)
+        ar = eng.sdfp_generate(prompts, 0, 24)
+        assert out.tokens == ar.tokens
+        assert eng.sdfp_generate(prompts[1:2], 4, 24).tokens[0] == out.tokens[1]
+        check_stream_against_oracle(m, prompts[0].tolist(), out.tokens[0])
+        # five rows at positions 320..324 against single rows, bit for bit, and against the oracle's logits
+        toks = si.make_prompts(shape.vocab, 1, 325, seed=63)[0].tolist()
+        for s0 in range(0, 320, 64):
+            eng.sdfp_forward_logits(toks[s0:s0 + 64], s0)
+        blk = eng.sdfp_forward_logits(toks[320:], 320)
+        one = np.concatenate([eng.sdfp_forward_logits(toks[i:i + 1], i) for i in range(320, 325)])
+        assert np.array_equal(one.view(np.uint32), blk.view(np.uint32))
+        ref = orc.CachedLM(m, max_seq=384).feed(toks, 0).numpy()[320:]
+        assert max(rel_l2(blk[r], ref[r]) for r in range(5)) < 1e-2
+    finally:
+        eng.close()
+
+
 def test_create_accepts_72_rows_and_rejects_more():
     w = si.weights_to(si.make_weights(si.TINY_BF16, (1, 2)), "cuda:0")
     with pytest.raises(pkg.SdfpError):
@@ -526,6 +552,33 @@ def test_wait_that_runs_out_returns_timeout(tiny_bf16):
     assert after.tokens == before.tokens and np.array_equal(after.stats, before.stats)
     ar = eng.sdfp_generate(prompt, 0, 24)
     assert ar.tokens == before.tokens
+
+
+def test_dense_path_wait_that_runs_out_returns_timeout():
+    """Failure path of the dense path's waits, without faulting anything: in the next forward call
+    the CTAs that hold the middle of a feature tile raise their flags where nobody looks, so the CTA
+    finishing the tile waits for a post that never comes, with a 20 ms limit.  The call must come back
+    quickly with SDFP_ETIMEOUT and the name of the wait, the kernels behind the one that gave up must do
+    nothing, and the context must work again afterwards (same logits, same tokens)."""
+    import time
+    eng, m, _ = make_pair(si.TINY_BF16, (1, 2), max_seq=96, max_batch=8, k_max=4)
+    try:
+        prompts = si.make_prompts(m.vocab, 8, 12, seed=71)
+        before = eng.sdfp_generate(prompts, 4, 16)
+        toks = prompts[0].tolist()
+        logits_before = eng.sdfp_forward_logits(toks, 0)
+        eng.sdfp_debug_expire_next_wait(20_000_000)
+        t0 = time.perf_counter()
+        with pytest.raises(pkg.SdfpError) as ei:
+            eng.sdfp_forward_logits(toks, 0)
+        assert time.perf_counter() - t0 < 1.0
+        assert ei.value.code == -5 and "never posted" in str(ei.value)
+        assert np.array_equal(eng.sdfp_forward_logits(toks, 0).view(np.uint32), logits_before.view(np.uint32))
+        after = eng.sdfp_generate(prompts, 4, 16)   # the hook was for one forward call only
+        assert after.tokens == before.tokens and np.array_equal(after.stats, before.stats)
+        assert eng.sdfp_generate(prompts, 0, 16).tokens == before.tokens
+    finally:
+        eng.close()
 
 
 # ---- the prompt pass on the tcgen05 path -------------------------------------------------------------
