@@ -767,6 +767,40 @@ def test_kv_sharing_draft_batch_and_sampling():
         eng.close()
 
 
+def test_dense_path_sublayer_mask_and_kv_sharing():
+    """The two draft variants on a context whose passes run on the dense path (8 sequence slots):
+    a sub-layer mask whose draft stack has an attention-only and an FFN-only layer (draft logits
+    against the oracle with the same two lists), and the draft attending the target's cache.
+    Tokens stay the target's in a batch with ragged acceptance; each sequence equals its solo run."""
+    shape = si.TINY_BF16
+    skip_attn, skip_ffn = (1, 2), (2,)
+    pkg.build_library()
+    w = si.make_weights(shape, skip_attn, skip_ffn=skip_ffn)
+    m = orc.Model.from_shape(shape, si.weights_to(w, "cpu"))
+    eng = pkg.Sdfp(shape, si.weights_to(w, "cuda:0"), max_seq=128, max_batch=8, k_max=4)
+    try:
+        ka, kf = si.keep_mask(shape.n_layers, skip_attn), si.keep_mask(shape.n_layers, skip_ffn)
+        eng.sdfp_set_draft_sublayers(ka, kf)
+        la, lf = orc.keep_layers(shape.n_layers, skip_attn), orc.keep_layers(shape.n_layers, skip_ffn)
+        toks = si.make_prompts(shape.vocab, 1, 40, seed=84)[0].tolist()
+        got = np.concatenate([eng.sdfp_forward_logits(toks[:17], 0, draft=True), eng.sdfp_forward_logits(toks[17:], 17, draft=True)])
+        ref = orc.CachedLM(m, la, max_seq=64, ffn_layers=lf).feed(toks, 0).numpy()
+        assert max(rel_l2(got[r], ref[r]) for r in range(40)) < 1e-2
+        prompts = si.make_prompts(shape.vocab, 8, 30, seed=85)
+        ar = eng.sdfp_generate(prompts, 0, 24)
+        for share in (False, True):
+            eng.sdfp_set_draft_kv_sharing(share)
+            out = eng.sdfp_generate(prompts, 4, 24)
+            assert out.tokens == ar.tokens
+            assert len({int(x) for x in out.stats[:, :, 1].ravel()}) > 1      # acceptance is ragged
+            for b in (0, 5):
+                assert eng.sdfp_generate(prompts[b:b + 1], 4, 24).tokens[0] == out.tokens[b]
+        check_stream_against_oracle(m, prompts[3].tolist(), ar.tokens[3])
+    finally:
+        eng.sdfp_set_draft_kv_sharing(False)
+        eng.close()
+
+
 def test_bf16_error_budget_against_unrounded_cache(tiny_bf16, l7b4, capsys):
     """The bf16 configurations round K/V to bf16 on both sides (oracle and library).  Against an
     oracle that keeps K/V in fp32 the library's logits must still sit inside the same tolerance;
